@@ -1,0 +1,222 @@
+"""Float64 CPU oracle of the FAEDKV / IWDFT hot path -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes wrapper over ``faedkv_oracle.c`` (plain C, compiled with gcc).  It
+is imported by the tests, by the smoke check and by the benchmark's CPU-baseline
+leg, and by nothing else; it shares no code with the CUDA path and does not
+import it.
+
+All arrays are float64 numpy arrays.  One "unit" is the ``[T, d]`` real matrix
+of one (batch, kv head, K-or-V); its compressed state is two ``[M, d]`` planes
+(real, imaginary) over the retained one-sided bins.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "faedkv_oracle.c")
+_LIB_DIR = os.path.join(_HERE, "_build")
+_LIB = os.path.join(_LIB_DIR, "libfaedkv_oracle.so")
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc -O2 -fopenmp; returns the library path."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    os.makedirs(_LIB_DIR, exist_ok=True)
+    tmp = _LIB + ".tmp.%d" % os.getpid()
+    cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
+           "-ffp-contract=off", _SRC, "-o", tmp, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+_f64p = ctypes.POINTER(ctypes.c_double)
+_i32p = ctypes.POINTER(ctypes.c_int32)
+_u8p = ctypes.POINTER(ctypes.c_uint8)
+_int = ctypes.c_int
+_i64 = ctypes.c_int64
+_u64 = ctypes.c_uint64
+_f64 = ctypes.c_double
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = ctypes.CDLL(build())
+    sig = {
+        "orc_weight": (_f64, [_int, _int]),
+        "orc_plan": (_int, [_int, _u8p, _i32p]),
+        "orc_fold_two_sided": (None, [_int, _u8p, _u8p]),
+        "orc_mask_lowpass": (_int, [_int, _int, _u8p]),
+        "orc_mask_mixed": (_int, [_int, _int, _int, _u64, _u8p]),
+        "orc_compress": (None, [_f64p, _int, _int, _int, _i32p, _int, _i64, _f64p, _f64p]),
+        "orc_compress_units": (None, [_f64p, _int, _int, _int, _int, _i32p, _int, _i64, _f64p, _f64p]),
+        "orc_append": (None, [_f64p, _f64p, _int, _int, _int, _i32p, _i64, _f64p]),
+        "orc_reconstruct": (None, [_f64p, _f64p, _int, _int, _int, _i32p, _int, _f64p]),
+        "orc_attention_dense": (None, [_f64p, _int, _f64p, _f64p, _int, _int, _f64, _f64p]),
+        "orc_decode_attn": (None, [_f64p, _int, _f64p, _f64p, _f64p, _f64p, _int, _int, _int,
+                                   _i32p, _int, _f64, _f64p]),
+        "orc_rotating_frame_step": (None, [_f64p, _f64p, _int, _int, _int, _i32p, _f64p]),
+        "orc_sliding_window_step": (None, [_f64p, _f64p, _int, _int, _int, _i32p, _f64p, _f64p]),
+        "orc_running_mean_step": (None, [_f64p, _f64p, _int, _int, _int, _i32p, _i64, _f64p]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def _d(a):
+    assert a.dtype == np.float64 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(_f64p)
+
+
+def _i(a):
+    assert a.dtype == np.int32 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(_i32p)
+
+
+def _u(a):
+    assert a.dtype == np.uint8 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(_u8p)
+
+
+def _f64arr(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def set_threads(n: int) -> None:
+    """Limit the OpenMP team used by the oracle (for the 1-thread timing)."""
+    _load()
+    omp = ctypes.CDLL("libgomp.so.1")
+    omp.omp_set_num_threads(int(n))
+
+
+def weight(P: int, k: int) -> float:
+    return float(_load().orc_weight(P, k))
+
+
+def weights(P: int, bins: np.ndarray) -> np.ndarray:
+    return np.array([weight(P, int(k)) for k in bins], dtype=np.float64)
+
+
+def plan(P: int, mask: np.ndarray) -> np.ndarray:
+    """One-sided keep mask (length P//2+1) -> ascending retained bin indices."""
+    mask = np.ascontiguousarray(mask, dtype=np.uint8)
+    assert mask.shape == (P // 2 + 1,)
+    bins = np.zeros(P // 2 + 1, dtype=np.int32)
+    M = _load().orc_plan(P, _u(mask), _i(bins))
+    return bins[:M].copy()
+
+
+def fold_two_sided(P: int, mask2: np.ndarray) -> np.ndarray:
+    mask2 = np.ascontiguousarray(mask2, dtype=np.uint8)
+    assert mask2.shape == (P,)
+    out = np.zeros(P // 2 + 1, dtype=np.uint8)
+    _load().orc_fold_two_sided(P, _u(mask2), _u(out))
+    return out
+
+
+def mask_lowpass(P: int, M: int) -> np.ndarray:
+    out = np.zeros(P // 2 + 1, dtype=np.uint8)
+    if _load().orc_mask_lowpass(P, M, _u(out)) != 0:
+        raise ValueError("bad low-pass mask request")
+    return out
+
+
+def mask_mixed(P: int, M: int, layer: int, seed: int) -> np.ndarray:
+    out = np.zeros(P // 2 + 1, dtype=np.uint8)
+    if _load().orc_mask_mixed(P, M, layer, seed, _u(out)) != 0:
+        raise ValueError("bad mixed mask request")
+    return out
+
+
+def compress(x: np.ndarray, P: int, bins: np.ndarray, pos0: int = 0):
+    """Pruned DFT of x [..., T, d] along the token axis -> (Cre, Cim) [..., M, d]."""
+    x = _f64arr(x)
+    bins = np.ascontiguousarray(bins, dtype=np.int32)
+    lead, (T, d) = x.shape[:-2], x.shape[-2:]
+    U = int(np.prod(lead)) if lead else 1
+    M = bins.shape[0]
+    Cre = np.zeros((U, M, d), dtype=np.float64)
+    Cim = np.zeros((U, M, d), dtype=np.float64)
+    if U == 1:
+        _load().orc_compress(_d(x), T, d, P, _i(bins), M, pos0, _d(Cre), _d(Cim))
+    else:
+        _load().orc_compress_units(_d(x), U, T, d, P, _i(bins), M, pos0, _d(Cre), _d(Cim))
+    return Cre.reshape(*lead, M, d), Cim.reshape(*lead, M, d)
+
+
+def append(Cre: np.ndarray, Cim: np.ndarray, P: int, bins: np.ndarray, t: int, xnew: np.ndarray):
+    """In-place IWDFT update of one unit's [M, d] planes with the token at position t."""
+    bins = np.ascontiguousarray(bins, dtype=np.int32)
+    xnew = _f64arr(xnew)
+    M, d = Cre.shape
+    assert Cim.shape == (M, d) and xnew.shape == (d,) and bins.shape == (M,)
+    _load().orc_append(_d(Cre), _d(Cim), M, d, P, _i(bins), t, _d(xnew))
+
+
+def reconstruct(Cre: np.ndarray, Cim: np.ndarray, P: int, bins: np.ndarray, L: int) -> np.ndarray:
+    """Pruned inverse DFT of one unit's planes -> [L, d]."""
+    bins = np.ascontiguousarray(bins, dtype=np.int32)
+    Cre, Cim = _f64arr(Cre), _f64arr(Cim)
+    M, d = Cre.shape
+    out = np.zeros((L, d), dtype=np.float64)
+    _load().orc_reconstruct(_d(Cre), _d(Cim), M, d, P, _i(bins), L, _d(out))
+    return out
+
+
+def attention_dense(q: np.ndarray, Kt: np.ndarray, Vt: np.ndarray, scale: float) -> np.ndarray:
+    q, Kt, Vt = _f64arr(q), _f64arr(Kt), _f64arr(Vt)
+    G, d = q.shape
+    L = Kt.shape[0]
+    out = np.zeros((G, d), dtype=np.float64)
+    _load().orc_attention_dense(_d(q), G, _d(Kt), _d(Vt), L, d, scale, _d(out))
+    return out
+
+
+def decode_attn(q: np.ndarray, CKre, CKim, CVre, CVim, P: int, bins: np.ndarray, L: int,
+                scale: float | None = None) -> np.ndarray:
+    """q [G, d] (query heads of one kv head) against one kv head's planes -> [G, d]."""
+    bins = np.ascontiguousarray(bins, dtype=np.int32)
+    q = _f64arr(q)
+    CKre, CKim, CVre, CVim = map(_f64arr, (CKre, CKim, CVre, CVim))
+    G, d = q.shape
+    M = bins.shape[0]
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    out = np.zeros((G, d), dtype=np.float64)
+    _load().orc_decode_attn(_d(q), G, _d(CKre), _d(CKim), _d(CVre), _d(CVim), M, d, P,
+                            _i(bins), L, scale, _d(out))
+    return out
+
+
+def rotating_frame_step(Rre, Rim, P, bins, xnew):
+    bins = np.ascontiguousarray(bins, dtype=np.int32)
+    M, d = Rre.shape
+    _load().orc_rotating_frame_step(_d(Rre), _d(Rim), M, d, P, _i(bins), _d(_f64arr(xnew)))
+
+
+def sliding_window_step(Sre, Sim, P, bins, x_out, x_in):
+    bins = np.ascontiguousarray(bins, dtype=np.int32)
+    M, d = Sre.shape
+    _load().orc_sliding_window_step(_d(Sre), _d(Sim), M, d, P, _i(bins),
+                                    _d(_f64arr(x_out)), _d(_f64arr(x_in)))
+
+
+def running_mean_step(Sre, Sim, P, bins, t, xnew):
+    bins = np.ascontiguousarray(bins, dtype=np.int32)
+    M, d = Sre.shape
+    _load().orc_running_mean_step(_d(Sre), _d(Sim), M, d, P, _i(bins), t, _d(_f64arr(xnew)))
