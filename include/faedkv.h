@@ -1,0 +1,166 @@
+/*
+ * faedkv.h -- C ABI of the FAEDKV / IWDFT hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The library keeps an LLM KV cache compressed as the retained bins of its
+ * discrete Fourier transform along the token axis (FAEDKV, Sec. 4).  It owns
+ * three things and nothing else: the per-layer bin plan, small device tables
+ * derived from it, and a fixed scratch area sized at faedkv_create().  Every
+ * tensor, every coefficient plane and every token counter belongs to the
+ * caller.
+ *
+ * Conventions
+ *   P        DFT grid size (the paper's N / N_DFT), fixed at create time.
+ *   bins[]   ascending retained ONE-SIDED bin indices in [0, P/2]; M = count.
+ *            K/V are real, so bin k stands for the conjugate pair (k, P-k);
+ *            w_k = 1 for k = 0 and k = P/2 (P even), else 2.
+ *   coef     float32, layout [batch][n_kv_heads][2][M][head_dim]; plane 0 is
+ *            the real part, plane 1 the imaginary part; head_dim contiguous.
+ *            Coefficients are always float32, whatever kv_dtype is.
+ *   t_len    int32 [batch], tokens folded into each sequence so far.  One
+ *            counter array per layer (append advances it).
+ *   K, V     [batch][n_kv_heads][T][head_dim] contiguous, element type kv_dtype.
+ *   q, out   [batch][n_q_heads][head_dim], element type kv_dtype; query head g
+ *            reads kv head g / (n_q_heads / n_kv_heads).
+ *   stream   a cudaStream_t passed as void* (NULL = the default stream).
+ *
+ * Pointers are DEVICE pointers unless a comment says "host".  Tensor and
+ * coefficient pointers must be 16-byte aligned, t_len 4-byte aligned.  Calls
+ * validate their arguments on the
+ * host and enqueue work on `stream`; they do not synchronise and do not
+ * allocate.  Return value: 0 on success, a negative faedkv_status otherwise;
+ * faedkv_last_error() gives the text of the last failure on that context.
+ * There is no CPU fallback: what the kernels do not support is an error.
+ * A context must not be used from two host threads at once.
+ */
+#ifndef FAEDKV_H
+#define FAEDKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct faedkv_ctx faedkv_ctx; /* opaque */
+
+typedef enum { FAEDKV_F32 = 0, FAEDKV_BF16 = 1 } faedkv_dtype;
+
+typedef enum {
+    FAEDKV_OK = 0,
+    FAEDKV_ERR_INVALID_ARG = -1, /* NULL pointer, negative size, bad enum            */
+    FAEDKV_ERR_NOT_PLANNED = -2, /* layer has no plan yet                            */
+    FAEDKV_ERR_SHAPE = -3,       /* batch / length outside what the context was made for */
+    FAEDKV_ERR_UNSUPPORTED = -4, /* configuration the kernels do not implement       */
+    FAEDKV_ERR_ALIGN = -5,       /* device pointer not 16-byte aligned               */
+    FAEDKV_ERR_CUDA = -6,        /* a CUDA call failed; see faedkv_last_error()      */
+    FAEDKV_ERR_TIMEOUT = -7      /* a bounded device-side wait gave up (see faedkv_device_status) */
+} faedkv_status;
+
+/* How the prefill transform is evaluated (faedkv_config.prefill_mode). */
+typedef enum {
+    FAEDKV_PREFILL_AUTO = 0,  /* bf16 K/V: tensor-core path; float32 K/V: float32 SIMT path */
+    FAEDKV_PREFILL_SIMT = 1,  /* float32 FMA contraction, twiddles exact to float32     */
+    FAEDKV_PREFILL_UMMA = 2   /* tcgen05 tensor-core contraction, bf16 operands, float32 accumulate */
+} faedkv_prefill_mode;
+
+typedef struct {
+    int n_layers;      /* >= 1                                                     */
+    int n_kv_heads;    /* >= 1                                                     */
+    int n_q_heads;     /* multiple of n_kv_heads, at most 8 query heads per kv head */
+    int head_dim;      /* must be 128                                              */
+    int n_dft;         /* P >= 2; need not be a power of two                       */
+    int max_batch;     /* >= 1; sizes the scratch area                             */
+    int kv_dtype;      /* faedkv_dtype of K, V, q, out                             */
+    int prefill_mode;  /* faedkv_prefill_mode                                      */
+    int twiddle_terms; /* tensor-core prefill only: 1 = twiddles rounded to one bf16
+                          (rel. error ~1e-3), 2 = bf16 hi+lo pair (~1e-5, twice the
+                          MMA work); 0 = default (1)                                */
+} faedkv_config;
+
+/* Create a context on the CURRENT CUDA device.  Allocates the scratch area
+ * (a few floats per (batch, query head, position of the grid)).  host: cfg, out. */
+int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out);
+
+/* Free the context, its plans and its scratch.  NULL is allowed. */
+void faedkv_destroy(faedkv_ctx *ctx);
+
+/* Text of the last error on this context ("" if none).  The pointer stays
+ * valid until the next failing call or faedkv_destroy(). */
+const char *faedkv_last_error(const faedkv_ctx *ctx);
+
+/* Plan a layer: the pruning rule of Eq. 6 as a keep-list.  bin_mask (host,
+ * length P/2 + 1): nonzero = retain one-sided bin k and, implicitly, its
+ * mirror P-k.  Builds the ascending bin list and its device copy; replaces an
+ * earlier plan of the same layer (the caller must not have work of that layer
+ * in flight).  *n_bins_out (host, may be NULL) receives M.  M = 0 is an error. */
+int faedkv_plan(faedkv_ctx *ctx, int layer, const uint8_t *bin_mask, int *n_bins_out);
+
+/* Number of retained bins of a planned layer, or a negative status. */
+int faedkv_n_bins(const faedkv_ctx *ctx, int layer);
+
+/* Copy the layer's bin list to bins_out (host, room for M int32). */
+int faedkv_get_bins(const faedkv_ctx *ctx, int layer, int32_t *bins_out);
+
+/* Bytes of ONE coefficient tensor (K or V) of a planned layer at this batch:
+ * batch * n_kv_heads * 2 * M * head_dim * 4.  0 if the layer is not planned. */
+size_t faedkv_coef_bytes(const faedkv_ctx *ctx, int layer, int batch);
+
+/* Synthetic mask generators used by the tests and the benchmark in place of
+ * the paper's ablation-study selection (Sec. 3.2), which needs a model and a
+ * corpus.  mask_out: host, length P/2 + 1.
+ *   lowpass: bins 0 .. M-1.
+ *   mixed:   chunks of 16 bins; the lowest floor((M/2)/16)*16 bins, plus
+ *            (M - that)/16 further chunks picked by a Fisher-Yates shuffle of
+ *            the remaining chunks below P/2, driven by the 64-bit LCG
+ *            s <- s*6364136223846793005 + 1442695040888963407 (draw = s >> 33),
+ *            s0 = seed*2654435761 + layer.  M must be a multiple of 16. */
+int faedkv_mask_lowpass(int n_dft, int n_keep, uint8_t *mask_out);
+int faedkv_mask_mixed(int n_dft, int n_keep, int layer, uint64_t seed, uint8_t *mask_out);
+
+/* Prefill transform (Sec. 4.2.1; Eq. 4 restricted to the retained bins by Eq. 6):
+ *   coef[k, c] = sum_{n < T} x[n, c] * exp(-j*2*pi*bins[k]*n / P)
+ * for every (batch, kv head) of K and of V.  SETS coefK, coefV and
+ * t_len[b] = T for b < batch.  T >= 1 may be smaller than, equal to or larger
+ * than P (positions wrap modulo P). */
+int faedkv_compress_prefill(faedkv_ctx *ctx, int layer, const void *K, const void *V,
+                            int batch, int T, float *coefK, float *coefV,
+                            int32_t *t_len, void *stream);
+
+/* IWDFT update (Sec. 4.1 Eq. 9 in its unnormalised, start-referenced form;
+ * Sec. 4.2.2 Eq. 12): fold one new token per sequence into the coefficients
+ * with unit weight,
+ *   coef[k, c] += x_new[c] * exp(-j*2*pi*bins[k]*t / P),  t = t_len[b],
+ * then t_len[b] += 1.  k_new, v_new: [batch][n_kv_heads][head_dim].  Only the
+ * retained bins exist, which equals updating every bin and pruning again. */
+int faedkv_append(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new,
+                  int batch, float *coefK, float *coefV, int32_t *t_len, void *stream);
+
+/* Reconstruction (Sec. 4.2.2 Eq. 11; Eq. 5 with every pruned bin zero):
+ *   x~[n, c] = (1/P) * sum_k w_k * (Re coef[k,c]*cos(2*pi*bins[k]*n/P)
+ *                                   - Im coef[k,c]*sin(2*pi*bins[k]*n/P))
+ * written to K_out, V_out [batch][n_kv_heads][L][head_dim] (kv_dtype) for
+ * n < min(t_len[b], P); rows from there up to L are written as zero.
+ * 1 <= L <= P.  Either of (coefK, K_out) or (coefV, V_out) may be a NULL pair. */
+int faedkv_reconstruct(faedkv_ctx *ctx, int layer, const float *coefK, const float *coefV,
+                       const int32_t *t_len, int batch, int L, void *K_out, void *V_out,
+                       void *stream);
+
+/* Decode attention (Eq. 3 on the reconstruction of Eq. 11):
+ *   out[g] = softmax_n( scale * q[g] . K~[n] ) * V~,  n < min(t_len[b], P)
+ * evaluated in the frequency domain, without writing K~ or V~ to memory.
+ * scale = 0 means 1/sqrt(head_dim).  Uses the context's scratch area: two
+ * calls on the same context must not overlap on the GPU. */
+int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *coefK,
+                       const float *coefV, const int32_t *t_len, int batch, float scale,
+                       void *out, void *stream);
+
+/* Device-side status word of the context (host read; synchronises `stream`):
+ * 0, or a nonzero code left by a kernel whose bounded wait on an mbarrier gave
+ * up.  Such a kernel returns early instead of hanging; its output is invalid. */
+int faedkv_device_status(faedkv_ctx *ctx, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FAEDKV_H */

@@ -1,0 +1,482 @@
+// Host side of the FAEDKV C ABI: context, per-layer plans, argument checks and
+// kernel launches.  See include/faedkv.h for the contract of every call.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/faedkv.h"
+#include "common.cuh"
+#include "k_append.cuh"
+#include "k_attn.cuh"
+#include "k_dft_simt.cuh"
+#include "k_prefill_umma.cuh"
+
+using namespace faedkv;
+
+namespace {
+
+struct LayerPlan {
+    int M = 0;
+    std::vector<int32_t> bins;
+    int32_t *d_bins = nullptr;
+};
+
+}  // namespace
+
+struct faedkv_ctx {
+    faedkv_config cfg;
+    int device = 0;
+    int gq = 1;    // query heads per kv head
+    int hqp = 32;  // n_q_heads rounded up to a multiple of 32
+    int max_M = 0;
+    int out_slices_cap = 0;
+    std::vector<LayerPlan> plans;
+    // scratch (device)
+    float *Qf = nullptr, *Pf = nullptr, *S = nullptr, *tile_max = nullptr, *colmax = nullptr,
+          *partial = nullptr;
+    unsigned int *tick = nullptr;      // [n_layers] tickets of k_append
+    unsigned int *dev_status = nullptr;  // one word, set by a kernel whose bounded wait gave up
+    UmmaPrefillState umma;             // tensor maps etc. of the tensor-core prefill
+    std::string err;
+};
+
+namespace {
+
+int fail(faedkv_ctx *ctx, int code, const char *fmt, ...) {
+    if (ctx != nullptr) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof(buf), fmt, ap);
+        va_end(ap);
+        ctx->err = buf;
+    }
+    return code;
+}
+
+#define CUDA_TRY(ctx, expr)                                                                   \
+    do {                                                                                      \
+        cudaError_t e_ = (expr);                                                              \
+        if (e_ != cudaSuccess)                                                                \
+            return fail(ctx, FAEDKV_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+int check_layer(faedkv_ctx *ctx, int layer, const LayerPlan **plan) {
+    if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= ctx->cfg.n_layers)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
+    const LayerPlan &p = ctx->plans[layer];
+    if (p.M == 0) return fail(ctx, FAEDKV_ERR_NOT_PLANNED, "layer %d has no plan", layer);
+    *plan = &p;
+    return FAEDKV_OK;
+}
+
+int check_batch(faedkv_ctx *ctx, int batch) {
+    if (batch < 1 || batch > ctx->cfg.max_batch)
+        return fail(ctx, FAEDKV_ERR_SHAPE, "batch %d outside [1, max_batch=%d]", batch, ctx->cfg.max_batch);
+    return FAEDKV_OK;
+}
+
+int check_ptrs(faedkv_ctx *ctx, std::initializer_list<const void *> ptrs) {
+    for (const void *p : ptrs)
+        if (!aligned16(p)) return fail(ctx, FAEDKV_ERR_ALIGN, "device pointer %p is not 16-byte aligned", p);
+    return FAEDKV_OK;
+}
+
+int check_tlen(faedkv_ctx *ctx, const void *t_len) {
+    if (!aligned4(t_len)) return fail(ctx, FAEDKV_ERR_ALIGN, "t_len %p is not 4-byte aligned", t_len);
+    return FAEDKV_OK;
+}
+
+int launch_check(faedkv_ctx *ctx, const char *what) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, FAEDKV_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
+    return FAEDKV_OK;
+}
+
+int out_slices(const faedkv_ctx *ctx, int batch, int M) {
+    // enough CTAs to fill the GPU twice over, at least 64 bins per slice
+    const int units = batch * ctx->cfg.n_kv_heads;
+    int s = (2 * 148 + units - 1) / units;
+    int cap = (M + 63) / 64;
+    if (s > cap) s = cap;
+    if (s < 1) s = 1;
+    return s;
+}
+
+void free_scratch(faedkv_ctx *ctx) {
+    cudaFree(ctx->Qf); cudaFree(ctx->Pf); cudaFree(ctx->S);
+    cudaFree(ctx->tile_max); cudaFree(ctx->colmax); cudaFree(ctx->partial);
+    ctx->Qf = ctx->Pf = ctx->S = ctx->tile_max = ctx->colmax = ctx->partial = nullptr;
+}
+
+// (Re)size the parts of the scratch area that depend on the largest M planned so far.
+int ensure_scratch(faedkv_ctx *ctx, int M) {
+    const faedkv_config &c = ctx->cfg;
+    const size_t B = (size_t)c.max_batch, P = (size_t)c.n_dft, HQP = (size_t)ctx->hqp;
+    if (ctx->S == nullptr) {
+        const size_t n_tiles = (P + kTilePos - 1) / kTilePos;
+        CUDA_TRY(ctx, cudaMalloc(&ctx->S, B * P * HQP * sizeof(float)));
+        CUDA_TRY(ctx, cudaMalloc(&ctx->tile_max, B * n_tiles * HQP * sizeof(float)));
+        CUDA_TRY(ctx, cudaMalloc(&ctx->colmax, B * HQP * sizeof(float)));
+    }
+    if (M > ctx->max_M) {
+        cudaFree(ctx->Qf); cudaFree(ctx->Pf); cudaFree(ctx->partial);
+        ctx->Qf = ctx->Pf = ctx->partial = nullptr;
+        CUDA_TRY(ctx, cudaMalloc(&ctx->Qf, B * 2 * (size_t)M * HQP * sizeof(float)));
+        CUDA_TRY(ctx, cudaMalloc(&ctx->Pf, B * 2 * (size_t)M * HQP * sizeof(float)));
+        // the slice count never exceeds 2*148 (units >= 1), nor ceil(M/64)
+        int cap = (M + 63) / 64;
+        if (cap > 2 * 148) cap = 2 * 148;
+        ctx->out_slices_cap = cap;
+        CUDA_TRY(ctx, cudaMalloc(&ctx->partial, B * c.n_kv_heads * (size_t)cap * ctx->gq * kHeadDim * sizeof(float)));
+        ctx->max_M = M;
+    }
+    return FAEDKV_OK;
+}
+
+__global__ void k_set_tlen(int32_t *t_len, int batch, int T) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < batch) t_len[i] = T;
+}
+
+template <typename TIn>
+int launch_prefill_simt(faedkv_ctx *ctx, const LayerPlan &p, const void *K, const void *V, int batch,
+                        int T, float *coefK, float *coefV, cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    DftUnitArgs a{};
+    a.x[0] = K; a.x[1] = V;
+    a.y[0] = coefK; a.y[1] = coefV;
+    a.x_unit = (long long)T * kHeadDim;
+    a.y_unit = 2LL * p.M * kHeadDim;
+    a.y_plane = (long long)p.M * kHeadDim;
+    a.x_row = kHeadDim; a.y_row = kHeadDim; a.col_blocks = 1;
+    dim3 grid((p.M + kTileBins - 1) / kTileBins, batch * c.n_kv_heads, 2);
+    k_dft_forward_simt<TIn, kHeadDim, false><<<grid, kSimtThreads, 0, st>>>(
+        a, p.d_bins, p.M, (uint32_t)c.n_dft, T, nullptr, 1, 0u, -1.0f, 0, nullptr);
+    return launch_check(ctx, "k_dft_forward_simt");
+}
+
+template <typename TOut>
+int launch_reconstruct(faedkv_ctx *ctx, const LayerPlan &p, const float *coefK, const float *coefV,
+                       const int32_t *t_len, int batch, int L, void *K_out, void *V_out, cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    DftUnitArgs a{};
+    int nt = 0;
+    if (coefK != nullptr) { a.x[nt] = K_out; a.y[nt] = const_cast<float *>(coefK); ++nt; }
+    if (coefV != nullptr) { a.x[nt] = V_out; a.y[nt] = const_cast<float *>(coefV); ++nt; }
+    a.x_unit = (long long)L * kHeadDim;
+    a.y_unit = 2LL * p.M * kHeadDim;
+    a.y_plane = (long long)p.M * kHeadDim;
+    a.x_row = kHeadDim; a.y_row = kHeadDim; a.col_blocks = 1;
+    dim3 grid((L + kTilePos - 1) / kTilePos, batch * c.n_kv_heads, nt);
+    k_dft_inverse_simt<TOut, kHeadDim><<<grid, kSimtThreads, 0, st>>>(
+        a, p.d_bins, p.M, (uint32_t)c.n_dft, L, t_len, c.n_kv_heads, 1.0f / (float)c.n_dft, nullptr);
+    return launch_check(ctx, "k_dft_inverse_simt");
+}
+
+template <typename TQ, int GQ>
+int launch_attn(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const float *coefK,
+                const float *coefV, const int32_t *t_len, int batch, float scale, void *out,
+                cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    const int H = c.n_kv_heads, HQ = c.n_q_heads, HQP = ctx->hqp, M = p.M, P = c.n_dft;
+    const int col_blocks = HQP / 32;
+    constexpr int KB = 16 / GQ;
+    // (1) query spectrum
+    {
+        dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
+        k_attn_qf<TQ, GQ><<<grid, kAttnWarps * 32, 0, st>>>(static_cast<const TQ *>(q), coefK, ctx->Qf, M, H, HQ, HQP);
+        if (int r = launch_check(ctx, "k_attn_qf")) return r;
+    }
+    // (2) scores over positions, with per-tile column maxima
+    const int n_tiles = (P + kTilePos - 1) / kTilePos;
+    {
+        DftUnitArgs a{};
+        a.x[0] = ctx->S; a.y[0] = ctx->Qf;
+        a.x_unit = (long long)P * HQP;
+        a.y_unit = 2LL * M * HQP;
+        a.y_plane = (long long)M * HQP;
+        a.x_row = HQP; a.y_row = HQP; a.col_blocks = col_blocks;
+        dim3 grid(n_tiles, batch * col_blocks, 1);
+        k_dft_inverse_simt<float, 32><<<grid, kSimtThreads, 0, st>>>(
+            a, p.d_bins, M, (uint32_t)P, P, t_len, 1, scale / (float)P, ctx->tile_max);
+        if (int r = launch_check(ctx, "k_dft_inverse_simt(scores)")) return r;
+        k_colmax<<<batch * col_blocks, 32, 0, st>>>(ctx->tile_max, n_tiles, 32, ctx->colmax);
+        if (int r = launch_check(ctx, "k_colmax")) return r;
+    }
+    // (3)+(4) softmax fused into the forward transform of the probabilities
+    {
+        DftUnitArgs a{};
+        a.x[0] = ctx->S; a.y[0] = ctx->Pf;
+        a.x_unit = (long long)P * HQP;
+        a.y_unit = 2LL * M * HQP;
+        a.y_plane = (long long)M * HQP;
+        a.x_row = HQP; a.y_row = HQP; a.col_blocks = col_blocks;
+        dim3 grid((M + kTileBins - 1) / kTileBins, batch * col_blocks, 1);
+        k_dft_forward_simt<float, 32, true><<<grid, kSimtThreads, 0, st>>>(
+            a, p.d_bins, M, (uint32_t)P, 0, t_len, 1, 0u, 1.0f, 0, ctx->colmax);
+        if (int r = launch_check(ctx, "k_dft_forward_simt(probabilities)")) return r;
+    }
+    // (5) value stream
+    {
+        const int slices = out_slices(ctx, batch, M);
+        const int per = (M + slices - 1) / slices;
+        dim3 grid(slices, batch * H);
+        k_attn_out<GQ><<<grid, kAttnWarps * 32, 0, st>>>(coefV, ctx->Pf, p.d_bins, ctx->partial, M, H, HQP, (uint32_t)P, per);
+        if (int r = launch_check(ctx, "k_attn_out")) return r;
+        k_attn_out_reduce<TQ><<<batch * H * GQ, kHeadDim, 0, st>>>(ctx->partial, static_cast<TQ *>(out), slices, GQ, 1.0f / (float)P);
+        if (int r = launch_check(ctx, "k_attn_out_reduce")) return r;
+    }
+    return FAEDKV_OK;
+}
+
+template <typename TQ>
+int dispatch_attn(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const float *coefK,
+                  const float *coefV, const int32_t *t_len, int batch, float scale, void *out,
+                  cudaStream_t st) {
+    switch (ctx->gq) {
+        case 1: return launch_attn<TQ, 1>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 2: return launch_attn<TQ, 2>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 4: return launch_attn<TQ, 4>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 8: return launch_attn<TQ, 8>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+    }
+    return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be 1, 2, 4 or 8");
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+extern "C" {
+
+int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
+    if (cfg == nullptr || out == nullptr) return FAEDKV_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->n_layers < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads < 1 || cfg->max_batch < 1 ||
+        cfg->n_dft < 2 || cfg->n_dft > (1 << 24))
+        return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->kv_dtype != FAEDKV_F32 && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->prefill_mode < FAEDKV_PREFILL_AUTO || cfg->prefill_mode > FAEDKV_PREFILL_UMMA) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->twiddle_terms < 0 || cfg->twiddle_terms > 2) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->head_dim != kHeadDim) return FAEDKV_ERR_UNSUPPORTED;
+    if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FAEDKV_ERR_UNSUPPORTED;
+    const int gq = cfg->n_q_heads / cfg->n_kv_heads;
+    if (gq != 1 && gq != 2 && gq != 4 && gq != 8) return FAEDKV_ERR_UNSUPPORTED;
+    if (cfg->prefill_mode == FAEDKV_PREFILL_UMMA && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_UNSUPPORTED;
+
+    faedkv_ctx *ctx = new (std::nothrow) faedkv_ctx();
+    if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;
+    ctx->cfg = *cfg;
+    ctx->gq = gq;
+    ctx->hqp = (cfg->n_q_heads + 31) / 32 * 32;
+    ctx->plans.resize(cfg->n_layers);
+    if (cudaGetDevice(&ctx->device) != cudaSuccess ||
+        cudaMalloc(&ctx->tick, sizeof(unsigned int) * (cfg->n_layers + 1)) != cudaSuccess ||
+        cudaMemset(ctx->tick, 0, sizeof(unsigned int) * (cfg->n_layers + 1)) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return FAEDKV_ERR_CUDA;
+    }
+    ctx->dev_status = ctx->tick + cfg->n_layers;
+    *out = ctx;
+    return FAEDKV_OK;
+}
+
+void faedkv_destroy(faedkv_ctx *ctx) {
+    if (ctx == nullptr) return;
+    for (LayerPlan &p : ctx->plans) cudaFree(p.d_bins);
+    free_scratch(ctx);
+    cudaFree(ctx->tick);
+    delete ctx;
+}
+
+const char *faedkv_last_error(const faedkv_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int faedkv_plan(faedkv_ctx *ctx, int layer, const uint8_t *bin_mask, int *n_bins_out) {
+    if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;
+    if (bin_mask == nullptr) return fail(ctx, FAEDKV_ERR_INVALID_ARG, "bin_mask is NULL");
+    if (layer < 0 || layer >= ctx->cfg.n_layers)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, ctx->cfg.n_layers);
+    const int n1 = ctx->cfg.n_dft / 2 + 1;
+    std::vector<int32_t> bins;
+    bins.reserve(n1);
+    for (int k = 0; k < n1; ++k)
+        if (bin_mask[k] != 0) bins.push_back(k);
+    if (bins.empty()) return fail(ctx, FAEDKV_ERR_INVALID_ARG, "mask of layer %d retains no bin", layer);
+    if (int r = ensure_scratch(ctx, (int)bins.size())) return r;
+    LayerPlan &p = ctx->plans[layer];
+    int32_t *d = nullptr;
+    CUDA_TRY(ctx, cudaMalloc(&d, bins.size() * sizeof(int32_t)));
+    cudaError_t e = cudaMemcpy(d, bins.data(), bins.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(d);
+        return fail(ctx, FAEDKV_ERR_CUDA, "upload of the bin list failed: %s", cudaGetErrorString(e));
+    }
+    cudaFree(p.d_bins);
+    p.d_bins = d;
+    p.M = (int)bins.size();
+    p.bins.swap(bins);
+    if (n_bins_out != nullptr) *n_bins_out = p.M;
+    return FAEDKV_OK;
+}
+
+int faedkv_n_bins(const faedkv_ctx *ctx, int layer) {
+    if (ctx == nullptr || layer < 0 || layer >= ctx->cfg.n_layers) return FAEDKV_ERR_INVALID_ARG;
+    if (ctx->plans[layer].M == 0) return FAEDKV_ERR_NOT_PLANNED;
+    return ctx->plans[layer].M;
+}
+
+int faedkv_get_bins(const faedkv_ctx *ctx, int layer, int32_t *bins_out) {
+    if (ctx == nullptr || bins_out == nullptr || layer < 0 || layer >= ctx->cfg.n_layers) return FAEDKV_ERR_INVALID_ARG;
+    const LayerPlan &p = ctx->plans[layer];
+    if (p.M == 0) return FAEDKV_ERR_NOT_PLANNED;
+    std::memcpy(bins_out, p.bins.data(), sizeof(int32_t) * p.M);
+    return FAEDKV_OK;
+}
+
+size_t faedkv_coef_bytes(const faedkv_ctx *ctx, int layer, int batch) {
+    if (ctx == nullptr || layer < 0 || layer >= ctx->cfg.n_layers || batch < 1) return 0;
+    const LayerPlan &p = ctx->plans[layer];
+    return (size_t)batch * ctx->cfg.n_kv_heads * 2 * (size_t)p.M * kHeadDim * sizeof(float);
+}
+
+int faedkv_mask_lowpass(int n_dft, int n_keep, uint8_t *mask_out) {
+    if (mask_out == nullptr || n_dft < 2) return FAEDKV_ERR_INVALID_ARG;
+    const int n1 = n_dft / 2 + 1;
+    if (n_keep < 0 || n_keep > n1) return FAEDKV_ERR_INVALID_ARG;
+    std::memset(mask_out, 0, n1);
+    std::memset(mask_out, 1, n_keep);
+    return FAEDKV_OK;
+}
+
+int faedkv_mask_mixed(int n_dft, int n_keep, int layer, uint64_t seed, uint8_t *mask_out) {
+    constexpr int kChunk = 16;
+    if (mask_out == nullptr || n_dft < 2 || n_keep <= 0 || n_keep % kChunk != 0) return FAEDKV_ERR_INVALID_ARG;
+    const int n1 = n_dft / 2 + 1;
+    const int low_chunks = (n_keep / 2) / kChunk;        // always-kept low chunks
+    const int extra_chunks = n_keep / kChunk - low_chunks;  // drawn chunks
+    const int pool_end = (n_dft / 2) / kChunk;           // chunks wholly below P/2
+    std::vector<int> pool;
+    for (int c = low_chunks; c < pool_end; ++c) pool.push_back(c);
+    if ((int)pool.size() < extra_chunks) return FAEDKV_ERR_INVALID_ARG;
+    std::memset(mask_out, 0, n1);
+    std::memset(mask_out, 1, (size_t)low_chunks * kChunk);
+    uint64_t state = seed * 2654435761ULL + (uint64_t)layer;
+    for (int i = 0; i < extra_chunks; ++i) {
+        state = state * 6364136223846793005ULL + 1442695040888963407ULL;
+        const uint64_t remaining = (uint64_t)(pool.size() - i);
+        std::swap(pool[i], pool[i + (size_t)((state >> 33) % remaining)]);
+        std::memset(mask_out + (size_t)pool[i] * kChunk, 1, kChunk);
+    }
+    return FAEDKV_OK;
+}
+
+int faedkv_compress_prefill(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch,
+                            int T, float *coefK, float *coefV, int32_t *t_len, void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    if (K == nullptr || V == nullptr || coefK == nullptr || coefV == nullptr || t_len == nullptr)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_compress_prefill");
+    if (T < 1) return fail(ctx, FAEDKV_ERR_SHAPE, "T = %d must be >= 1", T);
+    if (int r = check_ptrs(ctx, {K, V, coefK, coefV})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const faedkv_config &c = ctx->cfg;
+    int mode = c.prefill_mode;
+    if (mode == FAEDKV_PREFILL_AUTO)
+        mode = (c.kv_dtype == FAEDKV_BF16 && umma_prefill_available()) ? FAEDKV_PREFILL_UMMA : FAEDKV_PREFILL_SIMT;
+    int r;
+    if (mode == FAEDKV_PREFILL_UMMA) {
+        char msg[256] = {0};
+        r = umma_prefill_launch(ctx->umma, K, V, batch, c.n_kv_heads, T, p->d_bins, p->M, c.n_dft,
+                                c.twiddle_terms == 2 ? 2 : 1, coefK, coefV, ctx->dev_status, st, msg, sizeof(msg));
+        if (r != 0) return fail(ctx, r, "%s", msg);
+    } else if (c.kv_dtype == FAEDKV_BF16) {
+        r = launch_prefill_simt<__nv_bfloat16>(ctx, *p, K, V, batch, T, coefK, coefV, st);
+    } else {
+        r = launch_prefill_simt<float>(ctx, *p, K, V, batch, T, coefK, coefV, st);
+    }
+    if (r) return r;
+    k_set_tlen<<<(batch + 127) / 128, 128, 0, st>>>(t_len, batch, T);
+    return launch_check(ctx, "k_set_tlen");
+}
+
+int faedkv_append(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new, int batch,
+                  float *coefK, float *coefV, int32_t *t_len, void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    if (k_new == nullptr || v_new == nullptr || coefK == nullptr || coefV == nullptr || t_len == nullptr)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_append");
+    if (int r = check_ptrs(ctx, {k_new, v_new, coefK, coefV})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const faedkv_config &c = ctx->cfg;
+    dim3 grid((p->M + kAppendWarps - 1) / kAppendWarps, batch);
+    if (c.kv_dtype == FAEDKV_BF16)
+        k_append<__nv_bfloat16><<<grid, kAppendWarps * 32, 0, st>>>(
+            static_cast<const __nv_bfloat16 *>(k_new), static_cast<const __nv_bfloat16 *>(v_new), coefK, coefV,
+            t_len, p->d_bins, p->M, c.n_kv_heads, (uint32_t)c.n_dft, ctx->tick + layer);
+    else
+        k_append<float><<<grid, kAppendWarps * 32, 0, st>>>(
+            static_cast<const float *>(k_new), static_cast<const float *>(v_new), coefK, coefV, t_len,
+            p->d_bins, p->M, c.n_kv_heads, (uint32_t)c.n_dft, ctx->tick + layer);
+    return launch_check(ctx, "k_append");
+}
+
+int faedkv_reconstruct(faedkv_ctx *ctx, int layer, const float *coefK, const float *coefV,
+                       const int32_t *t_len, int batch, int L, void *K_out, void *V_out, void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    if (t_len == nullptr) return fail(ctx, FAEDKV_ERR_INVALID_ARG, "t_len is NULL");
+    if ((coefK == nullptr) != (K_out == nullptr) || (coefV == nullptr) != (V_out == nullptr) ||
+        (coefK == nullptr && coefV == nullptr))
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "coefficient / output pointers must come in non-NULL pairs");
+    if (L < 1 || L > ctx->cfg.n_dft) return fail(ctx, FAEDKV_ERR_SHAPE, "L = %d outside [1, P=%d]", L, ctx->cfg.n_dft);
+    if (int r = check_ptrs(ctx, {coefK, coefV, K_out, V_out})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->cfg.kv_dtype == FAEDKV_BF16)
+        return launch_reconstruct<__nv_bfloat16>(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);
+    return launch_reconstruct<float>(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);
+}
+
+int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *coefK, const float *coefV,
+                       const int32_t *t_len, int batch, float scale, void *out, void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    if (q == nullptr || coefK == nullptr || coefV == nullptr || t_len == nullptr || out == nullptr)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_decode_attn");
+    if (!(scale >= 0.0f)) return fail(ctx, FAEDKV_ERR_INVALID_ARG, "scale must be >= 0");
+    if (int r = check_ptrs(ctx, {q, coefK, coefV, out})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    if (scale == 0.0f) scale = 1.0f / sqrtf((float)ctx->cfg.head_dim);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->cfg.kv_dtype == FAEDKV_BF16)
+        return dispatch_attn<__nv_bfloat16>(ctx, *p, q, coefK, coefV, t_len, batch, scale, out, st);
+    return dispatch_attn<float>(ctx, *p, q, coefK, coefV, t_len, batch, scale, out, st);
+}
+
+int faedkv_device_status(faedkv_ctx *ctx, void *stream) {
+    if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned int w = 0;
+    CUDA_TRY(ctx, cudaMemcpyAsync(&w, ctx->dev_status, sizeof(w), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(ctx, cudaStreamSynchronize(st));
+    if (w != 0) {
+        fail(ctx, FAEDKV_ERR_TIMEOUT, "device status word = 0x%x (a bounded wait gave up)", w);
+        return (int)w;
+    }
+    return 0;
+}
+
+}  // extern "C"

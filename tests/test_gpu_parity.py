@@ -1,0 +1,367 @@
+"""GPU parity: every call of the C ABI against the float64 oracle on the same seeded inputs.
+
+Small cases are compared element by element; they span several tiles of every
+kernel plus ragged tails (bin counts, token counts, head counts that are not
+multiples of the tile sizes), both storage types, wrap-around positions, and
+the degenerate masks (a single bin, all bins).
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import (ATTN_MAX_ABS, REL_L2_BF16, REL_L2_F32, oracle_append, oracle_compress,
+                     oracle_decode_attn, oracle_reconstruct, rel_l2, to_np64)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def fk():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2507_20030_b200 import binding, build
+    build.build()
+    binding.load()
+    return binding
+
+
+def _tol(dtype):
+    return REL_L2_F32 if dtype == torch.float32 else REL_L2_BF16
+
+
+def _kvd(fk, dtype):
+    return fk.F32 if dtype == torch.float32 else fk.BF16
+
+
+def _mask_from_bins(P, bins):
+    m = np.zeros(P // 2 + 1, dtype=np.uint8)
+    m[np.asarray(bins)] = 1
+    return m
+
+
+def _random_mask(P, M, seed):
+    rng = np.random.default_rng(seed)
+    bins = np.sort(rng.choice(P // 2 + 1, size=M, replace=False))
+    return _mask_from_bins(P, bins)
+
+
+def _make(seed, B, H, T, dtype, pos0=0):
+    from paper_2507_20030_b200 import synth
+    K, V = synth.make_kv(seed, B, H, T, 128, pos0=pos0, dtype=dtype, device="cpu")
+    return K, V
+
+
+# ----------------------------------------------------------------------------- plan
+@pytest.mark.parametrize("P,M", [(64, 5), (100, 51), (2048, 256)])
+def test_plan_bins_bit_exact(fk, oracle, P, M):
+    ctx = fk.Context(n_layers=3, n_kv_heads=2, n_q_heads=2, n_dft=P, max_batch=1, kv_dtype=fk.F32)
+    for layer in range(3):
+        mask = _random_mask(P, M, 100 + layer)
+        assert ctx.plan(layer, mask) == M
+        got = ctx.get_bins(layer)
+        want = oracle.plan(P, mask)
+        assert got.dtype == np.int32 and got.tobytes() == want.tobytes()
+        assert ctx.coef_bytes(layer, 1) == 1 * 2 * 2 * M * 128 * 4
+    # re-planning a layer replaces its bins
+    mask = _random_mask(P, M, 999)
+    ctx.plan(0, mask)
+    assert ctx.get_bins(0).tobytes() == oracle.plan(P, mask).tobytes()
+    ctx.close()
+
+
+def test_error_codes(fk):
+    ctx = fk.Context(n_layers=2, n_kv_heads=2, n_q_heads=4, n_dft=64, max_batch=2, kv_dtype=fk.F32)
+    dev = "cuda"
+    K = torch.zeros(1, 2, 16, 128, device=dev)
+    coef = torch.zeros(1, 2, 2, 4, 128, device=dev)
+    t = torch.zeros(1, dtype=torch.int32, device=dev)
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx.compress_prefill(0, K, K, coef, coef, t)
+    assert e.value.code == -2                                   # not planned
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx.plan(0, np.zeros(33, dtype=np.uint8))
+    assert e.value.code == -1                                   # empty mask
+    ctx.plan(0, _mask_from_bins(64, [0, 1, 2, 5]))
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx.plan(5, _mask_from_bins(64, [0]))
+    assert e.value.code == -1                                   # layer out of range
+    K3 = torch.zeros(3, 2, 16, 128, device=dev)
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx.compress_prefill(0, K3, K3, coef, coef, t)
+    assert e.value.code == -3                                   # batch > max_batch
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx._check(ctx._lib.faedkv_compress_prefill(ctx._h, 0, K.data_ptr() + 4, K.data_ptr(), 1, 16,
+                                                    coef.data_ptr(), coef.data_ptr(), t.data_ptr(), None))
+    assert e.value.code == -5                                   # misaligned
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx._check(ctx._lib.faedkv_append(ctx._h, 0, None, K.data_ptr(), 1, coef.data_ptr(),
+                                          coef.data_ptr(), t.data_ptr(), None))
+    assert e.value.code == -1                                   # NULL tensor
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx.reconstruct(0, coef, coef, t, 65, K, K)
+    assert e.value.code == -3                                   # L > P
+    assert "outside" in str(e.value)
+    # the context is still usable after errors
+    ctx.compress_prefill(0, K, K, coef, coef, t)
+    torch.cuda.synchronize()
+    assert int(t[0]) == 16 and ctx.device_status() == 0
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- prefill
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,T,M,B,H", [(64, 64, 7, 1, 1), (100, 77, 51, 2, 3), (96, 250, 33, 1, 2),
+                                       (512, 512, 257, 1, 1)])
+def test_prefill_simt_matches_oracle(fk, oracle, dtype, P, T, M, B, H):
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                     prefill_mode=fk.PREFILL_SIMT)
+    mask = _random_mask(P, M, P + T)
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    K, V = _make(11 + P, B, H, T, dtype)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    torch.cuda.synchronize()
+    assert t_len.tolist() == [T] * B
+    assert rel_l2(to_np64(cK), oracle_compress(oracle, K, P, bins)) <= REL_L2_F32
+    assert rel_l2(to_np64(cV), oracle_compress(oracle, V, P, bins)) <= REL_L2_F32
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- append
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,M,B,H,steps", [(64, 33, 2, 3, 70), (1000, 77, 3, 8, 12), (256, 1, 1, 5, 5)])
+def test_append_matches_oracle(fk, oracle, dtype, P, M, B, H, steps):
+    from paper_2507_20030_b200 import synth
+    ctx = fk.Context(n_layers=2, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                     prefill_mode=fk.PREFILL_SIMT)
+    mask = _random_mask(P, M, 5 * P + M)
+    ctx.plan(1, mask)
+    bins = oracle.plan(P, mask)
+    rng = np.random.default_rng(3)
+    cK = torch.from_numpy(rng.standard_normal((B, H, 2, M, 128)).astype(np.float32)).cuda()
+    cV = torch.from_numpy(rng.standard_normal((B, H, 2, M, 128)).astype(np.float32)).cuda()
+    refK, refV = to_np64(cK), to_np64(cV)
+    t0 = np.array([0, P - 3, 5 * P + 1][:B], dtype=np.int32)       # ragged; wraps past P
+    t_len = torch.from_numpy(t0.copy()).cuda()
+    for s in range(steps):
+        k, v = synth.make_token(77, s, B, H, 128, pos=int(t0[0]) + s, dtype=dtype)
+        ctx.append(1, k.cuda(), v.cuda(), cK, cV, t_len)
+        oracle_append(oracle, refK, P, bins, t0 + s, k)
+        oracle_append(oracle, refV, P, bins, t0 + s, v)
+    torch.cuda.synchronize()
+    assert t_len.cpu().numpy().tolist() == (t0 + steps).tolist()
+    assert rel_l2(to_np64(cK), refK) <= REL_L2_F32
+    assert rel_l2(to_np64(cV), refV) <= REL_L2_F32
+    ctx.close()
+
+
+def test_appends_from_zero_equal_prefill(fk):
+    """T successive appends from the zero state reproduce the batch transform (float32 rounding apart)."""
+    from paper_2507_20030_b200 import synth
+    P, T, M, B, H = 128, 128, 40, 1, 2
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=fk.F32,
+                     prefill_mode=fk.PREFILL_SIMT)
+    ctx.plan(0, _random_mask(P, M, 1))
+    K, V = synth.make_kv(5, B, H, T, 128)
+    K, V = K.cuda(), V.cuda()
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K, V, cK, cV, t_len)
+    aK, aV = torch.zeros_like(cK), torch.zeros_like(cV)
+    t2 = torch.zeros(B, dtype=torch.int32, device="cuda")
+    for n in range(T):
+        ctx.append(0, K[:, :, n].contiguous(), V[:, :, n].contiguous(), aK, aV, t2)
+    torch.cuda.synchronize()
+    assert t2.tolist() == t_len.tolist() == [T]
+    assert rel_l2(to_np64(aK), to_np64(cK)) <= 1e-5
+    assert rel_l2(to_np64(aV), to_np64(cV)) <= 1e-5
+    ctx.close()
+
+
+def test_checkpoint_restore_is_bit_exact(fk):
+    """State is plain memory: append after a copy-out / copy-in equals the uninterrupted run."""
+    from paper_2507_20030_b200 import synth
+    P, M, B, H = 256, 48, 2, 4
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=fk.BF16,
+                     prefill_mode=fk.PREFILL_SIMT)
+    ctx.plan(0, fk.mask_mixed(P, M, 0, 9))
+    K, V = synth.make_kv(8, B, H, 200, 128, dtype=torch.bfloat16)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    toks = [synth.make_token(8, s, B, H, 128, pos=200 + s, dtype=torch.bfloat16) for s in range(6)]
+    for k, v in toks[:3]:
+        ctx.append(0, k.cuda(), v.cuda(), cK, cV, t_len)
+    saved = (cK.cpu().clone(), cV.cpu().clone(), t_len.cpu().clone())
+    for k, v in toks[3:]:
+        ctx.append(0, k.cuda(), v.cuda(), cK, cV, t_len)
+    rK, rV, rt = saved[0].cuda(), saved[1].cuda(), saved[2].cuda()
+    for k, v in toks[3:]:
+        ctx.append(0, k.cuda(), v.cuda(), rK, rV, rt)
+    torch.cuda.synchronize()
+    assert torch.equal(rK, cK) and torch.equal(rV, cV) and torch.equal(rt, t_len)
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- reconstruct
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,M,L,B,H,tl", [(64, 33, 64, 2, 1, [64, 40]), (100, 20, 77, 1, 3, [300]),
+                                          (512, 100, 512, 1, 2, [512]), (96, 1, 50, 1, 1, [96])])
+def test_reconstruct_matches_oracle(fk, oracle, dtype, P, M, L, B, H, tl):
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype))
+    mask = _random_mask(P, M, 9 * P + L) if M > 1 else _mask_from_bins(P, [0])
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    rng = np.random.default_rng(L)
+    cK = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * P ** 0.5).astype(np.float32)).cuda()
+    cV = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * P ** 0.5).astype(np.float32)).cuda()
+    t_np = np.array(tl, dtype=np.int32)
+    t_len = torch.from_numpy(t_np).cuda()
+    Ko = torch.full((B, H, L, 128), 7.0, dtype=dtype, device="cuda")
+    Vo = torch.full((B, H, L, 128), 7.0, dtype=dtype, device="cuda")
+    ctx.reconstruct(0, cK, cV, t_len, L, Ko, Vo)
+    torch.cuda.synchronize()
+    wantK = oracle_reconstruct(oracle, to_np64(cK), P, bins, t_np, L)
+    wantV = oracle_reconstruct(oracle, to_np64(cV), P, bins, t_np, L)
+    assert rel_l2(to_np64(Ko), wantK) <= _tol(dtype)
+    assert rel_l2(to_np64(Vo), wantV) <= _tol(dtype)
+    for b in range(B):                                           # rows past the live length are exactly zero
+        live = min(int(t_np[b]), P)
+        if live < L:
+            assert float(Ko[b, :, live:].abs().max()) == 0.0
+    # K only
+    Ko2 = torch.zeros_like(Ko)
+    ctx.reconstruct(0, cK, None, t_len, L, Ko2, None)
+    torch.cuda.synchronize()
+    assert torch.equal(Ko2, Ko)
+    ctx.close()
+
+
+def test_all_bins_round_trip(fk):
+    """All bins retained: reconstruct(compress(x)) returns x (float32)."""
+    P, B, H = 128, 1, 2
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=fk.F32,
+                     prefill_mode=fk.PREFILL_SIMT)
+    ctx.plan(0, np.ones(P // 2 + 1, dtype=np.uint8))
+    K, V = _make(2, B, H, P, torch.float32)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    Ko, Vo = torch.empty_like(K, device="cuda"), torch.empty_like(V, device="cuda")
+    ctx.reconstruct(0, cK, cV, t_len, P, Ko, Vo)
+    torch.cuda.synchronize()
+    assert rel_l2(to_np64(Ko), to_np64(K)) <= 1e-5
+    assert rel_l2(to_np64(Vo), to_np64(V)) <= 1e-5
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- decode attention
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,T,M,B,H,HQ,tl", [
+    (256, 256, 32, 2, 2, 8, None),        # GQA 4, full length
+    (200, 130, 37, 1, 3, 3, None),        # MHA (1 query head per kv head), t < P, odd sizes
+    (128, 128, 16, 2, 1, 8, [128, 70]),   # GQA 8, ragged lengths
+    (512, 512, 64, 1, 8, 32, None),       # 32 query heads, GQA 4
+    (128, 128, 24, 1, 20, 40, None),      # 40 query heads: two column blocks, GQA 2
+])
+def test_decode_attn_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, tl):
+    from paper_2507_20030_b200 import synth
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                     prefill_mode=fk.PREFILL_SIMT)
+    mask = _random_mask(P, M, 3 * P + M)
+    mask[0] = 1
+    M = int(mask.sum())
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    K, V = _make(21 + P, B, H, T, dtype)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    if tl is not None:
+        # shorter sequences: recompute their state from the first tl[b] tokens only
+        for b, t in enumerate(tl):
+            if t < T:
+                Kb, Vb = K[b:b + 1, :, :t].contiguous().cuda(), V[b:b + 1, :, :t].contiguous().cuda()
+                ctx.compress_prefill(0, Kb, Vb, cK[b:b + 1], cV[b:b + 1], t_len[b:b + 1])
+    q = synth.make_q(5, 0, B, HQ, 128, dtype=dtype)
+    out = torch.empty((B, HQ, 128), dtype=dtype, device="cuda")
+    ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out)
+    torch.cuda.synchronize()
+    t_np = t_len.cpu().numpy()
+    want = oracle_decode_attn(oracle, q, to_np64(cK), to_np64(cV), P, bins, t_np)
+    assert np.abs(to_np64(out) - want).max() <= ATTN_MAX_ABS
+    # explicit scale
+    out2 = torch.empty_like(out)
+    ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out2, scale=0.05)
+    torch.cuda.synchronize()
+    want2 = oracle_decode_attn(oracle, q, to_np64(cK), to_np64(cV), P, bins, t_np, scale=0.05)
+    assert np.abs(to_np64(out2) - want2).max() <= ATTN_MAX_ABS
+    ctx.close()
+
+
+def test_decode_attn_dc_only_is_mean_of_v(fk):
+    """Only bin 0 retained: the softmax is uniform and the output is the mean of V."""
+    P, B, H, HQ = 64, 1, 2, 8
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=fk.F32,
+                     prefill_mode=fk.PREFILL_SIMT)
+    ctx.plan(0, _mask_from_bins(P, [0]))
+    K, V = _make(4, B, H, P, torch.float32)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    q = torch.randn(B, HQ, 128, generator=torch.Generator().manual_seed(1))
+    out = torch.empty((B, HQ, 128), device="cuda")
+    ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out)
+    torch.cuda.synchronize()
+    want = V.double().mean(dim=2).repeat_interleave(HQ // H, dim=1).numpy()
+    assert np.abs(to_np64(out) - want).max() <= 1e-5
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- config 0, end to end
+def test_config0_end_to_end(fk, oracle):
+    """1 layer, B=1, 8 kv heads, d=128, T=2048 float32, low-pass M=256; 64 appends (positions wrap onto
+    slots 0..63); reconstruct L=2048; every tensor against the oracle."""
+    from paper_2507_20030_b200 import synth
+    P = T = 2048
+    M, B, H, HQ, steps = 256, 1, 8, 32, 64
+    seed = synth.config_seed(0, 0)
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=fk.F32)
+    mask = fk.mask_lowpass(P, M)
+    assert mask.tobytes() == oracle.mask_lowpass(P, M).tobytes()
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    assert ctx.get_bins(0).tobytes() == bins.tobytes()
+    K, V = synth.make_kv(seed, B, H, T, 128, dtype=torch.float32)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    torch.cuda.synchronize()
+    refK, refV = oracle_compress(oracle, K, P, bins), oracle_compress(oracle, V, P, bins)
+    assert rel_l2(to_np64(cK), refK) <= REL_L2_F32
+    assert rel_l2(to_np64(cV), refV) <= REL_L2_F32
+    for s in range(steps):
+        k, v = synth.make_token(seed, s, B, H, 128, pos=T + s, dtype=torch.float32)
+        ctx.append(0, k.cuda(), v.cuda(), cK, cV, t_len)
+        oracle_append(oracle, refK, P, bins, np.array([T + s]), k)
+        oracle_append(oracle, refV, P, bins, np.array([T + s]), v)
+    torch.cuda.synchronize()
+    assert t_len.tolist() == [T + steps]
+    assert rel_l2(to_np64(cK), refK) <= REL_L2_F32
+    assert rel_l2(to_np64(cV), refV) <= REL_L2_F32
+    Ko = torch.empty((B, H, P, 128), device="cuda")
+    Vo = torch.empty((B, H, P, 128), device="cuda")
+    ctx.reconstruct(0, cK, cV, t_len, P, Ko, Vo)
+    torch.cuda.synchronize()
+    t_np = np.array([T + steps])
+    assert rel_l2(to_np64(Ko), oracle_reconstruct(oracle, refK, P, bins, t_np, P)) <= REL_L2_F32
+    assert rel_l2(to_np64(Vo), oracle_reconstruct(oracle, refV, P, bins, t_np, P)) <= REL_L2_F32
+    q = synth.make_q(seed, 0, B, HQ, 128, dtype=torch.float32)
+    out = torch.empty((B, HQ, 128), device="cuda")
+    ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out)
+    torch.cuda.synchronize()
+    want = oracle_decode_attn(oracle, q, refK, refV, P, bins, t_np)
+    assert np.abs(to_np64(out) - want).max() <= ATTN_MAX_ABS
+    ctx.close()
