@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the FAEDKV / IWDFT hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--decode-iters D]
+
+One "step" is one pass of the whole hot path over one synthetic, Llama-3-8B-shaped cache (32 layers,
+8 kv heads / 32 query heads, head_dim 128, batch 1, T = P = 32768 bf16 tokens, per-layer mixed bin
+masks keeping 1/8 of the bins):
+
+    A. faedkv_compress_prefill of all 32 layers                      -> prefill tokens/s (the `value`)
+    B. D decode iterations of (faedkv_append + faedkv_decode_attn) on all 32 layers
+                                                                     -> decode us / layer / step
+    C. faedkv_reconstruct of all 32 layers (L = P)
+
+Inputs are resident in HBM before the timed region; every layer's tensors are distinct and the layers
+are cycled (4 GiB of K/V, 2 GiB of coefficients), so nothing survives in the 126 MB L2 between uses.
+`e2e` repeats phase A through the same C-ABI calls with the K/V in pinned HOST memory and the
+coefficients copied back to the host, copies inside the timed region.
+
+With N > 1 (torchrun) every rank runs the same workload on its own GPU: the path needs no
+inter-GPU exchange ("replicas only"), `value` is the sum over ranks, time the max over ranks.
+
+`--impl reference` times the float64 CPU oracle, as it stands, on the host cores on a bounded
+sample of the same workload and prints the same JSON line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "iwdft_prefill_tokens_per_s"
+UNIT = "tokens/s"
+
+WORKLOAD = dict(name="configs[1]: Llama-3-8B-shaped full cache, prefill 32768 tokens at 1/8 bin retention",
+                config=1, n_layers=32, n_kv_heads=8, n_q_heads=32, head_dim=128, batch=1, T=32768,
+                M=4096, mask="mixed")
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=float(d["hbm_gbs"]), bf16=float(d["bf16_tflops"]),
+                    bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# --------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        # the busiest half of the samples is "under load"
+        sm_sorted = sorted(sm)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_mhz_min": sm_sorted[0] if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------- reference arm
+def _oracle_units_seconds(orc, torch, synth, n_units, T, P, bins, seed):
+    """Time the oracle's pruned DFT of `n_units` units (kv heads of layer 0, K) over all retained bins."""
+    K, _ = synth.make_kv(seed, 1, n_units, T, 128, dtype=torch.bfloat16)
+    x = K[0].double().numpy()
+    t0 = time.perf_counter()
+    orc.compress(x, P, bins)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(target_s: float = 12.0) -> dict:
+    """Oracle prefill throughput on the host cores, from a bounded sample extrapolated over the
+    independent (layer, head, tensor) units of the workload."""
+    import torch
+    import oracle as orc
+    from paper_2507_20030_b200 import synth
+    orc.build()
+    W = WORKLOAD
+    P = T = W["T"]
+    cores = len(os.sched_getaffinity(0))
+    bins = orc.plan(P, orc.mask_mixed(P, W["M"], 0, synth.config_seed(W["config"])))
+    seed = synth.config_seed(W["config"], 0)
+    t1 = _oracle_units_seconds(orc, torch, synth, 1, T, P, bins, seed)
+    n_units = int(max(1, min(W["n_kv_heads"], round(target_s / t1))))
+    t_sample = t1 if n_units == 1 else _oracle_units_seconds(orc, torch, synth, n_units, T, P, bins, seed)
+    units = W["n_layers"] * W["batch"] * W["n_kv_heads"] * 2            # (layer, head, K|V)
+    full_s = t_sample * units / n_units
+    return {"value": W["batch"] * T / full_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": (f"pruned DFT of {n_units} of {units} units (layer 0, kv heads 0..{n_units - 1}, K): all {T} tokens "
+                       f"x 128 channels x {W['M']} bins in {t_sample:.2f} s; extrapolated linearly over units"),
+            "sample_seconds": t_sample}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    W = WORKLOAD
+    vals = []
+    base = None
+    for i in range(args.warmup + args.steps):
+        base = cpu_baseline(target_s=max(2.0, min(12.0, 90.0 / max(1, args.warmup + args.steps))))
+        if i >= args.warmup:
+            vals.append(base)
+    v = statistics.mean(b["value"] for b in vals)
+    ms = statistics.mean(W["batch"] * W["T"] / b["value"] for b in vals) * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": W["name"], "extrapolated": True},
+            "cpu_baseline": {**base, "value": v},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2507_20030_b200 import binding, build, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    peaks = _peaks()
+    W = WORKLOAD
+    NL, H, HQ, D, B, T, M = (W[k] for k in ("n_layers", "n_kv_heads", "n_q_heads", "head_dim", "batch", "T", "M"))
+    P = T
+    dev = torch.device("cuda", local)
+    ctx = binding.Context(n_layers=NL, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B,
+                          kv_dtype=binding.BF16, prefill_mode=args.prefill_mode,
+                          twiddle_terms=args.twiddle_terms)
+    base_seed = synth.config_seed(W["config"])
+    for l in range(NL):
+        ctx.plan(l, binding.mask_mixed(P, M, l, base_seed))
+
+    # ---- resident inputs and state
+    Ks, Vs, cKs, cVs, tls = [], [], [], [], []
+    for l in range(NL):
+        K, V = synth.make_kv(synth.config_seed(W["config"], l), B, H, T, D, dtype=torch.bfloat16, device=dev)
+        Ks.append(K); Vs.append(V)
+        cKs.append(ctx.alloc_coef(l, B, device=dev)); cVs.append(ctx.alloc_coef(l, B, device=dev))
+        tls.append(torch.zeros(B, dtype=torch.int32, device=dev))
+    n_dec = args.decode_iters
+    k_new = [synth.make_token(base_seed, s, B, H, D, pos=T + s, dtype=torch.bfloat16, device=dev) for s in range(n_dec)]
+    q_new = [synth.make_q(base_seed, s, B, HQ, D, dtype=torch.bfloat16, device=dev) for s in range(n_dec)]
+    attn_out = torch.empty((B, HQ, D), dtype=torch.bfloat16, device=dev)
+    Ko = torch.empty((B, H, P, D), dtype=torch.bfloat16, device=dev)
+    Vo = torch.empty_like(Ko)
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(record):
+        """One pass of the hot path. `record`: dict of lists of (start, stop) event pairs, or None."""
+        def timed(key, fn):
+            if record is None:
+                fn()
+                return
+            a, b = ev(), ev()
+            a.record(stream); fn(); b.record(stream)
+            record.setdefault(key, []).append((a, b))
+        for l in range(NL):
+            timed("prefill", lambda: ctx.compress_prefill(l, Ks[l], Vs[l], cKs[l], cVs[l], tls[l]))
+        for s in range(n_dec):
+            for l in range(NL):
+                timed("append", lambda: ctx.append(l, k_new[s][0], k_new[s][1], cKs[l], cVs[l], tls[l]))
+                timed("attn", lambda: ctx.decode_attn(l, q_new[s], cKs[l], cVs[l], tls[l], attn_out))
+        for l in range(NL):
+            timed("reconstruct", lambda: ctx.reconstruct(l, cKs[l], cVs[l], tls[l], P, Ko, Vo))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step(None)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count()
+    rec = {}
+    t_start, t_stop = ev(), ev()
+    barrier()
+    t_start.record(stream)
+    for _ in range(args.steps):
+        step(rec)
+    t_stop.record(stream)
+    barrier()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    if ctx.device_status() != 0:
+        raise RuntimeError("a kernel reported a device-side timeout; the numbers are invalid")
+
+    def total_ms(key):
+        return sum(a.elapsed_time(b) for a, b in rec[key])
+
+    phase_ms = {k: total_ms(k) / args.steps for k in rec}
+    step_ms = t_start.elapsed_time(t_stop) / args.steps
+    prefill_ms = phase_ms["prefill"]
+
+    if world > 1:
+        t = torch.tensor([prefill_ms, step_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        prefill_ms, step_ms = float(t[0]), float(t[1])
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        hK = [torch.empty(Ks[0].shape, dtype=torch.bfloat16).pin_memory() for _ in range(NL)]
+        hV = [torch.empty(Vs[0].shape, dtype=torch.bfloat16).pin_memory() for _ in range(NL)]
+        hcK = [torch.empty(cKs[l].shape, dtype=torch.float32).pin_memory() for l in range(NL)]
+        hcV = [torch.empty(cVs[l].shape, dtype=torch.float32).pin_memory() for l in range(NL)]
+        for l in range(NL):
+            hK[l].copy_(Ks[l]); hV[l].copy_(Vs[l])
+        torch.cuda.synchronize()
+        copy_in, copy_out = torch.cuda.Stream(), torch.cuda.Stream()
+        sK = [torch.empty_like(Ks[0]) for _ in range(2)]
+        sV = [torch.empty_like(Vs[0]) for _ in range(2)]
+
+        def e2e_step():
+            in_done = [None, None]
+            slot_free = [None, None]
+            for l in range(NL):
+                s = l & 1
+                with torch.cuda.stream(copy_in):
+                    if slot_free[s] is not None:
+                        copy_in.wait_event(slot_free[s])
+                    sK[s].copy_(hK[l], non_blocking=True)
+                    sV[s].copy_(hV[l], non_blocking=True)
+                    in_done[s] = copy_in.record_event()
+                stream.wait_event(in_done[s])
+                ctx.compress_prefill(l, sK[s], sV[s], cKs[l], cVs[l], tls[l])
+                done = stream.record_event()
+                slot_free[s] = done
+                with torch.cuda.stream(copy_out):
+                    copy_out.wait_event(done)
+                    hcK[l].copy_(cKs[l], non_blocking=True)
+                    hcV[l].copy_(cVs[l], non_blocking=True)
+            stream.wait_stream(copy_out)
+
+        h2d = sum(t.numel() * 2 for t in hK) + sum(t.numel() * 2 for t in hV)
+        d2h = sum(t.numel() * 4 for t in hcK) + sum(t.numel() * 4 for t in hcV)
+        e2e_step()
+        barrier()
+        k_e2e = max(1, min(args.steps, 3))
+        t0 = time.perf_counter()
+        a, b = ev(), ev()
+        a.record(stream)
+        for _ in range(k_e2e):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        wall_ms = (time.perf_counter() - t0) * 1e3 / k_e2e
+        e2e_ms = max(a.elapsed_time(b) / k_e2e, wall_ms if world == 1 else 0.0)
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t[0])
+        e2e = {"value": world * B * T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+               "what": "phase A through the C ABI with pinned host K/V in and host coefficient planes out"}
+        del hK, hV, hcK, hcV
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (prefill contraction), per launch (= one layer, K and V)
+    n_c = B * H * D
+    flop_per_launch = 2.0 * (2 * M) * T * n_c * 2            # 2*(2M)*T*N_c per tensor, K and V
+    prefill_launch_ms = total_ms("prefill") / len(rec["prefill"])
+    achieved_tf = flop_per_launch / (prefill_launch_ms * 1e-3) / 1e12
+    mode = "simt-f32" if args.prefill_mode == binding.PREFILL_SIMT else "tcgen05-bf16"
+    if mode == "tcgen05-bf16":
+        peak_tf, bound = peaks["bf16_sustained"], "tensor"
+    else:
+        # float32 FMA pipe: 148 SMs x 128 lanes x 2 FLOP x 1.965 GHz
+        peak_tf, bound = 148 * 128 * 2 * 1.965e9 / 1e12, "alu"
+    roofline = {"kernel": "prefill transform (" + mode + ")", "bound": bound, "achieved": achieved_tf,
+                "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf, "traffic": None,
+                "peak_source": peaks["source"] + (" bf16 sustained" if bound == "tensor" else " (derived f32 FMA peak)"),
+                "flop_per_launch": flop_per_launch, "launch_ms": prefill_launch_ms,
+                "mma_passes": (args.twiddle_terms if args.twiddle_terms else 1) if bound == "tensor" else None}
+
+    coef_bytes = 2 * B * H * 2 * M * D * 4                     # K and V planes of one layer
+    append_ms = total_ms("append") / len(rec["append"])
+    attn_ms = total_ms("attn") / len(rec["attn"])
+    recon_ms = total_ms("reconstruct") / len(rec["reconstruct"])
+    decode = {
+        "decode_us_per_layer_step": (append_ms + attn_ms) * 1e3,
+        "append": {"us": append_ms * 1e3, "bytes": 2 * coef_bytes, "bound": "hbm",
+                   "achieved": 2 * coef_bytes / (append_ms * 1e-3) / 1e9, "peak": peaks["hbm"], "unit": "GB/s",
+                   "frac": 2 * coef_bytes / (append_ms * 1e-3) / 1e9 / peaks["hbm"]},
+        "decode_attn": {"us": attn_ms * 1e3, "bytes": coef_bytes, "bound": "hbm",
+                        "achieved": coef_bytes / (attn_ms * 1e-3) / 1e9, "peak": peaks["hbm"], "unit": "GB/s",
+                        "frac": coef_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm"]},
+        "reconstruct": {"ms_per_layer": recon_ms, "flop": 2.0 * P * (2 * M) * n_c * 2,
+                        "achieved_tflops": 2.0 * P * (2 * M) * n_c * 2 / (recon_ms * 1e-3) / 1e12},
+        "decode_iters": n_dec,
+    }
+
+    line = {"metric": METRIC, "value": world * B * T / (prefill_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": W["name"], "n_layers": NL, "n_kv_heads": H, "n_q_heads": HQ, "head_dim": D,
+                       "batch": B, "T": T, "n_dft": P, "n_bins": M, "mask": "mixed (seeded, per layer)",
+                       "prefill_path": mode, "twiddle_terms": args.twiddle_terms or 1,
+                       "l2": "inputs larger than L2: 32 layers cycled, 128 MiB K/V + 64 MiB planes per layer",
+                       "multi_gpu": "replicas only"},
+            "phase_ms": phase_ms, "prefill_ms": prefill_ms,
+            "roofline": roofline, "decode": decode, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline()
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--decode-iters", type=int, default=2)
+    ap.add_argument("--prefill-mode", type=int, default=0, help="0 auto, 1 float32 SIMT, 2 tcgen05")
+    ap.add_argument("--twiddle-terms", type=int, default=0, help="tcgen05 prefill: 1 or 2 bf16 terms per twiddle")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -160,6 +160,10 @@ int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *c
  * up.  Such a kernel returns early instead of hanging; its output is invalid. */
 int faedkv_device_status(faedkv_ctx *ctx, void *stream);
 
+/* Number of kernels this context has enqueued since it was created (host
+ * counter; the benchmark reports its difference over the timed region). */
+unsigned long long faedkv_launch_count(const faedkv_ctx *ctx);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,7 +26,7 @@ EXPORTS = [
     "faedkv_create", "faedkv_destroy", "faedkv_last_error", "faedkv_plan", "faedkv_n_bins",
     "faedkv_get_bins", "faedkv_coef_bytes", "faedkv_mask_lowpass", "faedkv_mask_mixed",
     "faedkv_compress_prefill", "faedkv_append", "faedkv_reconstruct", "faedkv_decode_attn",
-    "faedkv_device_status",
+    "faedkv_device_status", "faedkv_launch_count",
 ]
 
 
@@ -85,6 +85,8 @@ def load() -> ctypes.CDLL:
     lib.faedkv_decode_attn.restype = _int
     lib.faedkv_device_status.argtypes = [_vp, _vp]
     lib.faedkv_device_status.restype = _int
+    lib.faedkv_launch_count.argtypes = [_vp]
+    lib.faedkv_launch_count.restype = ctypes.c_ulonglong
     _lib = lib
     return lib
 
@@ -217,6 +219,9 @@ class Context:
         self._check(self._lib.faedkv_decode_attn(
             self._h, layer, _ptr(q), _ptr(coefK), _ptr(coefV), _ptr(t_len), batch, float(scale),
             _ptr(out), _stream(stream)))
+
+    def launch_count(self) -> int:
+        return int(self._lib.faedkv_launch_count(self._h))
 
     def device_status(self, stream=None) -> int:
         return int(self._lib.faedkv_device_status(self._h, _stream(stream)))

@@ -40,6 +40,7 @@ struct faedkv_ctx {
     unsigned int *tick = nullptr;      // [n_layers] tickets of k_append
     unsigned int *dev_status = nullptr;  // one word, set by a kernel whose bounded wait gave up
     UmmaPrefillState umma;             // tensor maps etc. of the tensor-core prefill
+    unsigned long long launches = 0;   // kernels enqueued by this context so far
     std::string err;
 };
 
@@ -97,6 +98,7 @@ int check_tlen(faedkv_ctx *ctx, const void *t_len) {
 int launch_check(faedkv_ctx *ctx, const char *what) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, FAEDKV_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
+    ctx->launches += 1;
     return FAEDKV_OK;
 }
 
@@ -465,6 +467,8 @@ int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *c
         return dispatch_attn<__nv_bfloat16>(ctx, *p, q, coefK, coefV, t_len, batch, scale, out, st);
     return dispatch_attn<float>(ctx, *p, q, coefK, coefV, t_len, batch, scale, out, st);
 }
+
+unsigned long long faedkv_launch_count(const faedkv_ctx *ctx) { return ctx ? ctx->launches : 0ULL; }
 
 int faedkv_device_status(faedkv_ctx *ctx, void *stream) {
     if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;
