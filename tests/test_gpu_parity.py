@@ -365,3 +365,33 @@ def test_config0_end_to_end(fk, oracle):
     want = oracle_decode_attn(oracle, q, refK, refV, P, bins, t_np)
     assert np.abs(to_np64(out) - want).max() <= ATTN_MAX_ABS
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- tensor-core prefill
+@pytest.mark.parametrize("terms,tol", [(1, REL_L2_BF16), (2, REL_L2_F32)])
+@pytest.mark.parametrize("P,T,M,B,H", [
+    (512, 512, 128, 1, 1),      # one bin tile, 8 pipeline steps
+    (512, 512, 200, 1, 2),      # two bin tiles, ragged second tile
+    (1000, 700, 77, 2, 3),      # P not a power of two, T < P, ragged last token stage (700 = 10*64 + 60)
+    (256, 1000, 129, 1, 2),     # T > P: positions wrap
+    (2048, 2048, 256, 1, 8),    # config-0 shape in bf16
+    (64, 1, 3, 1, 1),           # a single token
+])
+def test_prefill_umma_matches_oracle(fk, oracle, terms, tol, P, T, M, B, H):
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=fk.BF16,
+                     prefill_mode=fk.PREFILL_UMMA, twiddle_terms=terms)
+    mask = _random_mask(P, M, 7 * P + T)
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    K, V = _make(31 + P + T, B, H, T, torch.bfloat16)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    cK.fill_(float("nan")); cV.fill_(float("nan"))
+    t_len = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    assert t_len.tolist() == [T] * B
+    errK = rel_l2(to_np64(cK), oracle_compress(oracle, K, P, bins))
+    errV = rel_l2(to_np64(cV), oracle_compress(oracle, V, P, bins))
+    assert errK <= tol and errV <= tol, (errK, errV)
+    ctx.close()
