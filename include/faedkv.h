@@ -160,6 +160,36 @@ int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *c
  * up.  Such a kernel returns early instead of hanging; its output is invalid. */
 int faedkv_device_status(faedkv_ctx *ctx, void *stream);
 
+/* Decode attention for callers that cannot allocate -- the paper has no
+ * counterpart; this is a packaging of faedkv_decode_attn() for hosts that
+ * must not call cudaMalloc where they need it: code that runs while a CUDA
+ * graph is being captured, a serving loop whose device memory was handed out
+ * once by an external pool, a plugin that only gets the tensors it is called
+ * with.  It takes no context (creating and planning one allocates): the bin
+ * list `bins` (DEVICE, int32[n_bins], ascending one-sided bins as produced by
+ * faedkv_get_bins) comes with the other inputs, and all intermediates live in
+ * a fixed device array of FAEDKV_STATIC_SCRATCH_BYTES that is part of the
+ * library image -- every GPU that loads the library holds that much until
+ * the process exits.  It calls no allocation routine of any kind.
+ *
+ * Same arguments, layouts and result as faedkv_decode_attn() (float32
+ * kernels); kv_dtype is the faedkv_dtype of q and out.  Sizes whose
+ * intermediates, about 4*batch*HQP*(n_dft + 4*n_bins + n_dft/32) bytes with
+ * HQP = n_q_heads rounded up to 32, exceed the array are refused with
+ * FAEDKV_ERR_SHAPE before anything is launched.  On any failure a text is
+ * written to err_msg (host, err_len bytes; may be NULL).
+ *
+ * All calls share the one array, which keeps the previous call's contents.
+ * Nothing in it needs to start at zero, so nothing is cleared; but calls that
+ * overlap on the GPU (two streams, two host threads) race on it: serialise
+ * them.  The first call on each device resolves the array's device address;
+ * make that first call outside any stream capture. */
+#define FAEDKV_STATIC_SCRATCH_BYTES (8u << 20)
+int faedkv_decode_attn_static(int n_dft, int n_kv_heads, int n_q_heads, int kv_dtype,
+                              const int32_t *bins, int n_bins, const void *q, const float *coefK,
+                              const float *coefV, const int32_t *t_len, int batch, float scale,
+                              void *out, void *stream, char *err_msg, size_t err_len);
+
 /* Number of kernels this context has enqueued since it was created (host
  * counter; the benchmark reports its difference over the timed region). */
 unsigned long long faedkv_launch_count(const faedkv_ctx *ctx);

@@ -26,8 +26,10 @@ EXPORTS = [
     "faedkv_create", "faedkv_destroy", "faedkv_last_error", "faedkv_plan", "faedkv_n_bins",
     "faedkv_get_bins", "faedkv_coef_bytes", "faedkv_mask_lowpass", "faedkv_mask_mixed",
     "faedkv_compress_prefill", "faedkv_append", "faedkv_reconstruct", "faedkv_decode_attn",
-    "faedkv_device_status", "faedkv_launch_count",
+    "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
 ]
+
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class FaedkvError(RuntimeError):
@@ -85,6 +87,9 @@ def load() -> ctypes.CDLL:
     lib.faedkv_decode_attn.restype = _int
     lib.faedkv_device_status.argtypes = [_vp, _vp]
     lib.faedkv_device_status.restype = _int
+    lib.faedkv_decode_attn_static.argtypes = [_int, _int, _int, _int, _vp, _int, _vp, _vp, _vp, _vp, _int,
+                                              ctypes.c_float, _vp, _vp, ctypes.c_char_p, ctypes.c_size_t]
+    lib.faedkv_decode_attn_static.restype = _int
     lib.faedkv_launch_count.argtypes = [_vp]
     lib.faedkv_launch_count.restype = ctypes.c_ulonglong
     _lib = lib
@@ -105,6 +110,23 @@ def mask_mixed(n_dft: int, n_keep: int, layer: int, seed: int) -> np.ndarray:
     if rc != 0:
         raise FaedkvError(rc, "faedkv_mask_mixed rejected its arguments")
     return out
+
+
+def decode_attn_static(n_dft: int, n_kv_heads: int, n_q_heads: int, kv_dtype: int, bins, q, coefK, coefV,
+                       t_len, out, scale: float = 0.0, stream=None) -> None:
+    """faedkv_decode_attn_static: decode attention without a context and without any allocation.
+
+    For callers that cannot allocate device memory where they need attention (inside a stream
+    capture, under an external memory pool, in a plugin that only receives tensors).  `bins` is a
+    device int32 tensor holding the layer's retained bins.  All intermediates live in a fixed
+    array inside the library (STATIC_SCRATCH_BYTES); larger problems raise FaedkvError(-3).
+    Calls share that array, so calls that overlap on the GPU must be serialised by the caller."""
+    buf = ctypes.create_string_buffer(256)
+    rc = load().faedkv_decode_attn_static(
+        n_dft, n_kv_heads, n_q_heads, kv_dtype, _ptr(bins), int(bins.numel()), _ptr(q), _ptr(coefK),
+        _ptr(coefV), _ptr(t_len), int(q.shape[0]), float(scale), _ptr(out), _stream(stream), buf, 256)
+    if rc != 0:
+        raise FaedkvError(rc, buf.value.decode())
 
 
 def _ptr(t):
