@@ -184,7 +184,10 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     build.build()
     peaks = _peaks()
-    W = WORKLOAD
+    W = dict(WORKLOAD)
+    if args.layers:
+        W["n_layers"] = args.layers
+        W["name"] += f" [first {args.layers} layers only: profiling case, not a bench value]"
     NL, H, HQ, D, B, T, M = (W[k] for k in ("n_layers", "n_kv_heads", "n_q_heads", "head_dim", "batch", "T", "M"))
     P = T
     dev = torch.device("cuda", local)
@@ -392,6 +395,9 @@ def main():
     ap.add_argument("--decode-iters", type=int, default=2)
     ap.add_argument("--prefill-mode", type=int, default=0, help="0 auto, 1 float32 SIMT, 2 tcgen05")
     ap.add_argument("--twiddle-terms", type=int, default=0, help="tcgen05 prefill: 1 or 2 bf16 terms per twiddle")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run only the first N layers of the workload (small case for profiler captures; "
+                         "a bench value must use the default = all layers)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
