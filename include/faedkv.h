@@ -64,6 +64,14 @@ typedef enum {
     FAEDKV_PREFILL_UMMA = 2   /* tcgen05 tensor-core contraction, bf16 operands, float32 accumulate */
 } faedkv_prefill_mode;
 
+/* How reconstruction and the two transforms inside decode attention are evaluated
+ * (faedkv_config.decode_mode). */
+typedef enum {
+    FAEDKV_DECODE_AUTO = 0,  /* bf16 tensors: tensor-core path; float32 tensors: float32 SIMT path */
+    FAEDKV_DECODE_SIMT = 1,  /* float32 FMA contractions, twiddles exact to float32            */
+    FAEDKV_DECODE_UMMA = 2   /* tcgen05 contractions with f16 operands, float32 accumulate (bf16 tensors only) */
+} faedkv_decode_mode;
+
 typedef struct {
     int n_layers;      /* >= 1                                                     */
     int n_kv_heads;    /* >= 1                                                     */
@@ -76,6 +84,7 @@ typedef struct {
     int twiddle_terms; /* tensor-core prefill only: 1 = twiddles rounded to one bf16
                           (rel. error ~1e-3), 2 = bf16 hi+lo pair (~1e-5, twice the
                           MMA work); 0 = default (1)                                */
+    int decode_mode;   /* faedkv_decode_mode                                       */
 } faedkv_config;
 
 /* Create a context on the CURRENT CUDA device.  Allocates the scratch area

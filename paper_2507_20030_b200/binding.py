@@ -21,6 +21,7 @@ LIB_PATH = os.path.join(_HERE, "lib", "libfaedkv.so")
 
 F32, BF16 = 0, 1
 PREFILL_AUTO, PREFILL_SIMT, PREFILL_UMMA = 0, 1, 2
+DECODE_AUTO, DECODE_SIMT, DECODE_UMMA = 0, 1, 2
 
 EXPORTS = [
     "faedkv_create", "faedkv_destroy", "faedkv_last_error", "faedkv_plan", "faedkv_n_bins",
@@ -41,7 +42,7 @@ class FaedkvError(RuntimeError):
 class Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "n_layers", "n_kv_heads", "n_q_heads", "head_dim", "n_dft", "max_batch", "kv_dtype",
-        "prefill_mode", "twiddle_terms")]
+        "prefill_mode", "twiddle_terms", "decode_mode")]
 
 
 _lib = None
@@ -158,11 +159,12 @@ class Context:
     head_dim: int = 128
     prefill_mode: int = PREFILL_AUTO
     twiddle_terms: int = 0
+    decode_mode: int = DECODE_AUTO
 
     def __post_init__(self):
         self._lib = load()
         cfg = Config(self.n_layers, self.n_kv_heads, self.n_q_heads, self.head_dim, self.n_dft,
-                     self.max_batch, self.kv_dtype, self.prefill_mode, self.twiddle_terms)
+                     self.max_batch, self.kv_dtype, self.prefill_mode, self.twiddle_terms, self.decode_mode)
         h = _vp()
         rc = self._lib.faedkv_create(ctypes.byref(cfg), ctypes.byref(h))
         if rc != 0:

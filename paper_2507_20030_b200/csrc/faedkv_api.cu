@@ -13,6 +13,8 @@
 #include "k_attn.cuh"
 #include "k_dft_simt.cuh"
 #include "k_prefill_umma.cuh"
+#include "k_idft_umma.cuh"
+#include "k_attn_umma.cuh"
 
 using namespace faedkv;
 
@@ -22,6 +24,16 @@ struct LayerPlan {
     int M = 0;
     std::vector<int32_t> bins;
     int32_t *d_bins = nullptr;
+    float *d_tab = nullptr;   // [M][16] per-bin phasors e^{jwk i}, i = 1..8 (tensor-core inverse transform)
+};
+
+constexpr int kSplitsCap = 8;   // most position splits of the probability spectrum
+
+// Scratch of the tensor-core decode / reconstruct path (bf16 tensors only).
+struct TcScratch {
+    __half *Qf16 = nullptr, *P16 = nullptr, *C16K = nullptr, *C16V = nullptr;
+    float *S = nullptr, *tile_max = nullptr, *cmax = nullptr, *psum = nullptr, *colsum = nullptr, *PfS = nullptr;
+    int gtot_max = 0, max_M = 0;
 };
 
 }  // namespace
@@ -40,6 +52,8 @@ struct faedkv_ctx {
     unsigned int *tick = nullptr;      // [n_layers] tickets of k_append
     unsigned int *dev_status = nullptr;  // one word, set by a kernel whose bounded wait gave up
     UmmaPrefillState umma;             // tensor maps etc. of the tensor-core prefill
+    TcScratch tc;
+    bool use_tc = false;               // bf16 tensors and decode_mode != SIMT
     unsigned long long launches = 0;   // kernels enqueued by this context so far
     std::string err;
 };
@@ -116,6 +130,10 @@ void free_scratch(faedkv_ctx *ctx) {
     cudaFree(ctx->Qf); cudaFree(ctx->Pf); cudaFree(ctx->S);
     cudaFree(ctx->tile_max); cudaFree(ctx->colmax); cudaFree(ctx->partial);
     ctx->Qf = ctx->Pf = ctx->S = ctx->tile_max = ctx->colmax = ctx->partial = nullptr;
+    TcScratch &t = ctx->tc;
+    cudaFree(t.Qf16); cudaFree(t.P16); cudaFree(t.C16K); cudaFree(t.C16V); cudaFree(t.S); cudaFree(t.tile_max);
+    cudaFree(t.cmax); cudaFree(t.psum); cudaFree(t.colsum); cudaFree(t.PfS);
+    t = TcScratch();
 }
 
 // (Re)size the parts of the scratch area that depend on the largest M planned so far.
@@ -139,6 +157,185 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
         ctx->out_slices_cap = cap;
         CUDA_TRY(ctx, cudaMalloc(&ctx->partial, B * c.n_kv_heads * (size_t)cap * ctx->gq * kHeadDim * sizeof(float)));
         ctx->max_M = M;
+    }
+    if (ctx->use_tc) {
+        TcScratch &t = ctx->tc;
+        if (t.S == nullptr) {
+            t.gtot_max = (c.max_batch * c.n_q_heads + 63) / 64 * 64;
+            const size_t G = (size_t)t.gtot_max;
+            CUDA_TRY(ctx, cudaMalloc(&t.S, P * G * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&t.tile_max, ((P + 31) / 32) * G * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&t.cmax, G * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&t.colsum, G * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&t.psum, ((P + kSoftmaxRows - 1) / kSoftmaxRows) * G * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&t.P16, P * G * sizeof(__half)));
+        }
+        if (M > t.max_M) {
+            const size_t G = (size_t)t.gtot_max;
+            cudaFree(t.Qf16); cudaFree(t.PfS); cudaFree(t.C16K); cudaFree(t.C16V);
+            t.Qf16 = nullptr; t.PfS = nullptr; t.C16K = t.C16V = nullptr;
+            CUDA_TRY(ctx, cudaMalloc(&t.Qf16, 2 * (size_t)M * G * sizeof(__half)));
+            CUDA_TRY(ctx, cudaMemset(t.Qf16, 0, 2 * (size_t)M * G * sizeof(__half)));   // padded columns stay finite
+            CUDA_TRY(ctx, cudaMalloc(&t.PfS, (size_t)kSplitsCap * 2 * M * G * sizeof(float)));
+            const size_t cbytes = B * c.n_kv_heads * 2 * (size_t)M * kHeadDim * sizeof(__half);
+            CUDA_TRY(ctx, cudaMalloc(&t.C16K, cbytes));
+            CUDA_TRY(ctx, cudaMalloc(&t.C16V, cbytes));
+            t.max_M = M;
+        }
+    }
+    return FAEDKV_OK;
+}
+
+// 3-D tiled tensor map with 128-byte swizzle and zero fill outside the tensor.
+int make_map3(faedkv_ctx *ctx, CUtensorMap *map, const void *base, CUtensorMapDataType dt, size_t elem, uint64_t d0,
+              uint64_t d1, uint64_t d2, uint64_t stride1_elems, uint64_t stride2_elems, uint32_t b0, uint32_t b1) {
+    char msg[200];
+    if (int r = umma_resolve_encode(ctx->umma, msg, sizeof(msg))) return fail(ctx, r, "%s", msg);
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {stride1_elems * elem, stride2_elems * elem};
+    cuuint32_t box[3] = {b0, b1, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = ctx->umma.encode(map, dt, 3, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ctx, FAEDKV_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return FAEDKV_OK;
+}
+
+template <typename K>
+int opt_in_smem(faedkv_ctx *ctx, K kernel, uint32_t bytes) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) return fail(ctx, FAEDKV_ERR_CUDA, "cannot opt in to %u bytes of shared memory: %s", bytes, cudaGetErrorString(e));
+    return FAEDKV_OK;
+}
+
+template <int NCOLS, int NT, int MODE>
+int launch_idft(faedkv_ctx *ctx, const CUtensorMap &m0, const CUtensorMap &m1, const idft::Args &a, dim3 grid, cudaStream_t st) {
+    using C = idft::Cfg<NCOLS, NT>;
+    if (int r = opt_in_smem(ctx, k_idft_umma<NCOLS, NT, MODE>, C::kSmemBytes)) return r;
+    k_idft_umma<NCOLS, NT, MODE><<<grid, idft::kThreads, C::kSmemBytes, st>>>(m0, m1, a);
+    return launch_check(ctx, "k_idft_umma");
+}
+
+template <int NCOLS>
+int launch_pspec(faedkv_ctx *ctx, const CUtensorMap &mp, const LayerPlan &p, int P, int rows_per_split, int Gtot, dim3 grid,
+                 cudaStream_t st) {
+    using C = pspec::Cfg<NCOLS>;
+    if (int r = opt_in_smem(ctx, k_pspec_umma<NCOLS>, C::kSmemBytes)) return r;
+    k_pspec_umma<NCOLS><<<grid, pspec::kThreads, C::kSmemBytes, st>>>(mp, p.d_bins, p.M, (uint32_t)P, rows_per_split, Gtot,
+                                                                       ctx->tc.PfS, ctx->dev_status);
+    return launch_check(ctx, "k_pspec_umma");
+}
+
+// Reconstruction on tensor cores (bf16 outputs): convert the planes to scaled f16, then one inverse-transform launch.
+int launch_reconstruct_tc(faedkv_ctx *ctx, const LayerPlan &p, const float *coefK, const float *coefV, const int32_t *t_len,
+                          int batch, int L, void *K_out, void *V_out, cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    TcScratch &t = ctx->tc;
+    const int units = batch * c.n_kv_heads, M = p.M, P = c.n_dft;
+    const size_t n_vec = (size_t)units * 2 * M * kHeadDim / 8;
+    const float *src[2] = {coefK, coefV};
+    __half *dst[2] = {t.C16K, t.C16V};
+    CUtensorMap maps[2];
+    int nt = 0;
+    void *outs[2] = {nullptr, nullptr};
+    for (int i = 0; i < 2; ++i) {
+        if (src[i] == nullptr) continue;
+        k_coef_to_half<<<(unsigned)((n_vec + 255) / 256), 256, 0, st>>>(src[i], dst[nt], p.d_bins, M, (uint32_t)P, n_vec);
+        if (int r = launch_check(ctx, "k_coef_to_half")) return r;
+        if (int r = make_map3(ctx, &maps[nt], dst[nt], CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, kHeadDim, (uint64_t)M,
+                              (uint64_t)units * 2, kHeadDim, (uint64_t)M * kHeadDim, 64, idft::kBinsPerStage))
+            return r;
+        outs[nt] = (i == 0) ? K_out : V_out;
+        ++nt;
+    }
+    idft::Args a{};
+    a.bins = p.d_bins; a.tab = p.d_tab; a.t_len = t_len; a.M = M; a.P = (uint32_t)P; a.Lrows = L;
+    a.outK = outs[0]; a.outV = outs[1]; a.H = c.n_kv_heads; a.status = ctx->dev_status;
+    if (nt == 2) {
+        dim3 grid((L + 255) / 256, units);
+        return launch_idft<256, 2, 0>(ctx, maps[0], maps[1], a, grid, st);
+    }
+    dim3 grid((L + 255) / 256, units);
+    return launch_idft<128, 2, 0>(ctx, maps[0], maps[0], a, grid, st);
+}
+
+template <typename TQ, int GQ>
+int launch_attn_tc(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const float *coefK, const float *coefV,
+                   const int32_t *t_len, int batch, float scale, void *out, cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    TcScratch &t = ctx->tc;
+    const int H = c.n_kv_heads, HQ = c.n_q_heads, M = p.M, P = c.n_dft;
+    const int n_cols = batch * HQ;
+    const int Gtot = (n_cols + 63) / 64 * 64;
+    const int ncols = (Gtot % 256 == 0) ? 256 : (Gtot % 128 == 0) ? 128 : 64;
+    const int col_blocks = Gtot / ncols;
+    constexpr int KB = 16 / GQ;
+    // (1) scaled query spectrum in f16
+    {
+        dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
+        k_attn_qf16<TQ, GQ><<<grid, kAttnWarps * 32, 0, st>>>(static_cast<const TQ *>(q), coefK, p.d_bins, t.Qf16, M, H, HQ,
+                                                              Gtot, (uint32_t)P, scale / (float)P);
+        if (int r = launch_check(ctx, "k_attn_qf16")) return r;
+    }
+    // (2) scores
+    {
+        CUtensorMap mq;
+        if (int r = make_map3(ctx, &mq, t.Qf16, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)Gtot, (uint64_t)M, 2,
+                              (uint64_t)Gtot, (uint64_t)M * Gtot, 64, idft::kBinsPerStage))
+            return r;
+        idft::Args a{};
+        a.bins = p.d_bins; a.tab = p.d_tab; a.t_len = t_len; a.M = M; a.P = (uint32_t)P; a.Lrows = P;
+        a.S = t.S; a.tile_max = t.tile_max; a.Gtot = Gtot; a.HQ = HQ; a.n_seq_cols = n_cols; a.status = ctx->dev_status;
+        const int tiles2 = (P + 255) / 256;
+        const bool two = tiles2 * col_blocks >= 148;
+        dim3 grid(two ? tiles2 : (P + 127) / 128, col_blocks);
+        int r;
+        if (ncols == 256) r = two ? launch_idft<256, 2, 1>(ctx, mq, mq, a, grid, st) : launch_idft<256, 1, 1>(ctx, mq, mq, a, grid, st);
+        else if (ncols == 128) r = two ? launch_idft<128, 2, 1>(ctx, mq, mq, a, grid, st) : launch_idft<128, 1, 1>(ctx, mq, mq, a, grid, st);
+        else r = two ? launch_idft<64, 2, 1>(ctx, mq, mq, a, grid, st) : launch_idft<64, 1, 1>(ctx, mq, mq, a, grid, st);
+        if (r) return r;
+    }
+    // (3) softmax numerators in f16 + normalisers
+    const int n_groups = (P + 31) / 32, n_sblocks = (P + kSoftmaxRows - 1) / kSoftmaxRows;
+    {
+        k_colmax_par<<<Gtot / 32, 256, 0, st>>>(t.tile_max, n_groups, Gtot, t.cmax);
+        if (int r = launch_check(ctx, "k_colmax_par")) return r;
+        dim3 grid(n_sblocks, Gtot / 64);
+        k_softmax_half<<<grid, 256, 0, st>>>(t.S, t.cmax, t_len, t.P16, t.psum, P, Gtot, HQ, n_cols);
+        if (int r = launch_check(ctx, "k_softmax_half")) return r;
+        k_colsum<<<Gtot / 32, 32, 0, st>>>(t.psum, n_sblocks, Gtot, t.colsum);
+        if (int r = launch_check(ctx, "k_colsum")) return r;
+    }
+    // (4) probability spectrum, positions split over CTAs
+    const int bin_tiles = (M + 127) / 128;
+    int splits = (2 * 148 + bin_tiles * col_blocks - 1) / (bin_tiles * col_blocks);
+    if (splits > kSplitsCap) splits = kSplitsCap;
+    if (splits > (P + 511) / 512) splits = (P + 511) / 512;
+    if (splits < 1) splits = 1;
+    const int rows_per_split = ((P + splits - 1) / splits + 63) / 64 * 64;
+    {
+        CUtensorMap mp;
+        if (int r = make_map3(ctx, &mp, t.P16, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, (uint64_t)Gtot, (uint64_t)P, 1, (uint64_t)Gtot,
+                              (uint64_t)P * Gtot, 64, pspec::kTileTok))
+            return r;
+        dim3 grid(bin_tiles, col_blocks, splits);
+        int r;
+        if (ncols == 256) r = launch_pspec<256>(ctx, mp, p, P, rows_per_split, Gtot, grid, st);
+        else if (ncols == 128) r = launch_pspec<128>(ctx, mp, p, P, rows_per_split, Gtot, grid, st);
+        else r = launch_pspec<64>(ctx, mp, p, P, rows_per_split, Gtot, grid, st);
+        if (r) return r;
+    }
+    // (5) value stream
+    {
+        const int slices = out_slices(ctx, batch, M);
+        const int per = (M + slices - 1) / slices;
+        dim3 grid(slices, batch * H);
+        k_attn_out2<GQ><<<grid, kAttnWarps * 32, 0, st>>>(coefV, t.PfS, p.d_bins, ctx->partial, M, H, HQ, Gtot, splits, (uint32_t)P, per);
+        if (int r = launch_check(ctx, "k_attn_out2")) return r;
+        k_attn_out_reduce2<TQ><<<batch * H * GQ, kHeadDim, 0, st>>>(ctx->partial, t.colsum, static_cast<TQ *>(out), slices, GQ,
+                                                                   1.0f / (float)P);
+        if (int r = launch_check(ctx, "k_attn_out_reduce2")) return r;
     }
     return FAEDKV_OK;
 }
@@ -243,6 +440,14 @@ template <typename TQ>
 int dispatch_attn(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const float *coefK,
                   const float *coefV, const int32_t *t_len, int batch, float scale, void *out,
                   cudaStream_t st) {
+    if (ctx->use_tc) {
+        switch (ctx->gq) {
+            case 1: return launch_attn_tc<TQ, 1>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+            case 2: return launch_attn_tc<TQ, 2>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+            case 4: return launch_attn_tc<TQ, 4>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+            case 8: return launch_attn_tc<TQ, 8>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+        }
+    }
     switch (ctx->gq) {
         case 1: return launch_attn<TQ, 1>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
         case 2: return launch_attn<TQ, 2>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
@@ -266,6 +471,8 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     if (cfg->kv_dtype != FAEDKV_F32 && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->prefill_mode < FAEDKV_PREFILL_AUTO || cfg->prefill_mode > FAEDKV_PREFILL_UMMA) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->twiddle_terms < 0 || cfg->twiddle_terms > 2) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->decode_mode < FAEDKV_DECODE_AUTO || cfg->decode_mode > FAEDKV_DECODE_UMMA) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->decode_mode == FAEDKV_DECODE_UMMA && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->head_dim != kHeadDim) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FAEDKV_ERR_UNSUPPORTED;
     const int gq = cfg->n_q_heads / cfg->n_kv_heads;
@@ -277,6 +484,7 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     ctx->cfg = *cfg;
     ctx->gq = gq;
     ctx->hqp = (cfg->n_q_heads + 31) / 32 * 32;
+    ctx->use_tc = cfg->kv_dtype == FAEDKV_BF16 && cfg->decode_mode != FAEDKV_DECODE_SIMT;
     ctx->plans.resize(cfg->n_layers);
     if (cudaGetDevice(&ctx->device) != cudaSuccess ||
         cudaMalloc(&ctx->tick, sizeof(unsigned int) * (cfg->n_layers + 1)) != cudaSuccess ||
@@ -292,7 +500,7 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
 
 void faedkv_destroy(faedkv_ctx *ctx) {
     if (ctx == nullptr) return;
-    for (LayerPlan &p : ctx->plans) cudaFree(p.d_bins);
+    for (LayerPlan &p : ctx->plans) { cudaFree(p.d_bins); cudaFree(p.d_tab); }
     free_scratch(ctx);
     cudaFree(ctx->tick);
     delete ctx;
@@ -320,8 +528,25 @@ int faedkv_plan(faedkv_ctx *ctx, int layer, const uint8_t *bin_mask, int *n_bins
         cudaFree(d);
         return fail(ctx, FAEDKV_ERR_CUDA, "upload of the bin list failed: %s", cudaGetErrorString(e));
     }
+    float *tab = nullptr;
+    if (ctx->use_tc) {
+        e = cudaMalloc(&tab, bins.size() * 16 * sizeof(float));
+        if (e != cudaSuccess) {
+            cudaFree(d);
+            return fail(ctx, FAEDKV_ERR_CUDA, "allocation of the phasor table failed: %s", cudaGetErrorString(e));
+        }
+        const int n = (int)bins.size() * 8;
+        k_bin_tables<<<(n + 255) / 256, 256>>>(d, (int)bins.size(), (uint32_t)ctx->cfg.n_dft, tab);
+        e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) {
+            cudaFree(d); cudaFree(tab);
+            return fail(ctx, FAEDKV_ERR_CUDA, "building the phasor table failed: %s", cudaGetErrorString(e));
+        }
+    }
     cudaFree(p.d_bins);
+    cudaFree(p.d_tab);
     p.d_bins = d;
+    p.d_tab = tab;
     p.M = (int)bins.size();
     p.bins.swap(bins);
     if (n_bins_out != nullptr) *n_bins_out = p.M;
@@ -446,6 +671,7 @@ int faedkv_reconstruct(faedkv_ctx *ctx, int layer, const float *coefK, const flo
     if (int r = check_ptrs(ctx, {coefK, coefV, K_out, V_out})) return r;
     if (int r = check_tlen(ctx, t_len)) return r;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->use_tc) return launch_reconstruct_tc(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);
     if (ctx->cfg.kv_dtype == FAEDKV_BF16)
         return launch_reconstruct<__nv_bfloat16>(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);
     return launch_reconstruct<float>(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);

@@ -32,10 +32,11 @@
 #include <cstdio>
 
 #include "common.cuh"
+#include "umma_common.cuh"
 
 namespace faedkv {
 
-namespace umma {
+namespace prefill {
 
 constexpr int kTileBinsU = 128;   // bins per CTA (rows of each accumulator)
 constexpr int kTileTok = 64;      // tokens per pipeline stage (one 128-byte swizzle row of bf16)
@@ -45,7 +46,6 @@ constexpr int kThreads = (2 + kGenWarps) * 32;
 constexpr uint32_t kATileBytes = kTileBinsU * kTileTok * 2;   // 16 KB
 constexpr uint32_t kBTileBytes = kTileTok * kNCols * 2;       // 32 KB
 constexpr uint32_t kBoxBytes = kTileTok * 64 * 2;             // one TMA box: 64 tokens x 64 channels
-constexpr uint64_t kWaitLimitNs = 1000000000ull;              // one bounded wait gives up after ~1 s
 
 constexpr uint32_t kErrTimeoutTma = 0x11, kErrTimeoutGen = 0x12, kErrTimeoutMma = 0x13, kErrTimeoutEpi = 0x14;
 
@@ -55,117 +55,20 @@ template <int TERMS> struct Cfg {
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-// ---- PTX wrappers ------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_timer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: false when the phase did not complete within kWaitLimitNs.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    uint64_t t0 = 0;
-    for (uint32_t i = 0;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 255u) {
-            const uint64_t now = global_timer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
-        }
-    }
-}
-__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// Arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed.
-__device__ __forceinline__ void mma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptors (sm_100 format: version 1 at bit 46, 128-byte swizzle = 2 at bit 61).
-// K-major operand, rows of 128 bytes, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t desc_kmajor_sw128(uint32_t saddr) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-// MN-major operand: 64-element (128-byte) runs along MN, 8 K-rows per 1024-byte atom;
-// leading offset = distance between 64-element MN blocks, stride offset = between 8-row K groups.
-__device__ __forceinline__ uint64_t desc_mnmajor_sw128(uint32_t saddr, uint32_t mn_block_bytes) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(mn_block_bytes >> 4) << 16) |
-           ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
 // kind::f16 instruction descriptor: D float32, A and B bf16, A K-major, B MN-major, M = 128, N = 256.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                             ((uint32_t)(kNCols >> 3) << 17) | ((uint32_t)(kTileBinsU >> 4) << 24);
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
-}
-__device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
-
-}  // namespace umma
+}  // namespace prefill
 
 // grid = (ceil(M / 128), batch * H); block = 320; dynamic smem = Cfg<TERMS>::kSmemBytes
 template <int TERMS>
-__global__ void __launch_bounds__(umma::kThreads, 1)
+__global__ void __launch_bounds__(prefill::kThreads, 1)
 k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const int32_t *__restrict__ bins, int M, uint32_t P, int T, uint32_t pos0,
                float *__restrict__ coefK, float *__restrict__ coefV, unsigned int *__restrict__ status) {
     using namespace umma;
+    using namespace prefill;
     using C = Cfg<TERMS>;
     constexpr int S = C::kStages;
     extern __shared__ uint8_t smem_raw[];
@@ -387,20 +290,25 @@ inline bool umma_prefill_available() { return true; }
 
 // K/V [units][T][128] bf16 as a 3-D tensor map; box = 64 channels x 64 tokens x 1 unit, 128-byte swizzle.
 // Rows past T read as zero, so a ragged last stage adds nothing.
-inline int umma_make_map(UmmaPrefillState &st, CUtensorMap *map, const void *base, int units, int T, char *msg, size_t n) {
-    if (st.encode == nullptr) {
-        void *fn = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-        if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) {
-            snprintf(msg, n, "cuTensorMapEncodeTiled is not available from the driver");
-            return -6;
-        }
-        st.encode = reinterpret_cast<PFN_encodeTiled>(fn);
+// Resolve cuTensorMapEncodeTiled through the runtime (the library does not link libcuda).
+inline int umma_resolve_encode(UmmaPrefillState &st, char *msg, size_t n) {
+    if (st.encode != nullptr) return 0;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess) {
+        snprintf(msg, n, "cuTensorMapEncodeTiled is not available from the driver");
+        return -6;
     }
+    st.encode = reinterpret_cast<PFN_encodeTiled>(fn);
+    return 0;
+}
+
+inline int umma_make_map(UmmaPrefillState &st, CUtensorMap *map, const void *base, int units, int T, char *msg, size_t n) {
+    if (int r = umma_resolve_encode(st, msg, n)) return r;
     cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)T, (cuuint64_t)units};
     cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)T * kHeadDim * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)umma::kTileTok, 1};
+    cuuint32_t box[3] = {64, (cuuint32_t)prefill::kTileTok, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = st.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -416,7 +324,7 @@ template <int TERMS>
 inline int umma_launch_t(UmmaPrefillState &st, const CUtensorMap &mK, const CUtensorMap &mV, int units, int T,
                          const int32_t *d_bins, int M, int P, float *coefK, float *coefV, unsigned int *status,
                          cudaStream_t stream, char *msg, size_t n) {
-    using C = umma::Cfg<TERMS>;
+    using C = prefill::Cfg<TERMS>;
     if (!st.attr_set[TERMS]) {
         cudaError_t e = cudaFuncSetAttribute(k_prefill_umma<TERMS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
         if (e != cudaSuccess) {
@@ -425,8 +333,8 @@ inline int umma_launch_t(UmmaPrefillState &st, const CUtensorMap &mK, const CUte
         }
         st.attr_set[TERMS] = true;
     }
-    dim3 grid((M + umma::kTileBinsU - 1) / umma::kTileBinsU, units);
-    k_prefill_umma<TERMS><<<grid, umma::kThreads, C::kSmemBytes, stream>>>(mK, mV, d_bins, M, (uint32_t)P, T, 0u, coefK, coefV, status);
+    dim3 grid((M + prefill::kTileBinsU - 1) / prefill::kTileBinsU, units);
+    k_prefill_umma<TERMS><<<grid, prefill::kThreads, C::kSmemBytes, stream>>>(mK, mV, d_bins, M, (uint32_t)P, T, 0u, coefK, coefV, status);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         snprintf(msg, n, "launch of k_prefill_umma failed: %s", cudaGetErrorString(e));

@@ -68,7 +68,7 @@ def test_create_rejects_bad_configs_before_touching_cuda(lib):
     from paper_2507_20030_b200 import binding
     h = ctypes.c_void_p()
     good = dict(n_layers=1, n_kv_heads=8, n_q_heads=32, head_dim=128, n_dft=2048, max_batch=1,
-                kv_dtype=binding.F32, prefill_mode=0, twiddle_terms=0)
+                kv_dtype=binding.F32, prefill_mode=0, twiddle_terms=0, decode_mode=0)
     for key, bad, code in [("head_dim", 64, -4), ("n_dft", 1, -1), ("n_q_heads", 12, -4),
                            ("n_q_heads", 128, -4), ("kv_dtype", 7, -1), ("max_batch", 0, -1),
                            ("twiddle_terms", 3, -1), ("n_layers", 0, -1)]:
