@@ -67,9 +67,12 @@ typedef enum {
 /* How reconstruction and the two transforms inside decode attention are evaluated
  * (faedkv_config.decode_mode). */
 typedef enum {
-    FAEDKV_DECODE_AUTO = 0,  /* bf16 tensors: tensor-core path; float32 tensors: float32 SIMT path */
+    FAEDKV_DECODE_AUTO = 0,  /* P a power of two in [64, 2^19]: FFT-shaped transforms; otherwise
+                                bf16 tensors: tensor-core path; float32 tensors: float32 SIMT path */
     FAEDKV_DECODE_SIMT = 1,  /* float32 FMA contractions, twiddles exact to float32            */
-    FAEDKV_DECODE_UMMA = 2   /* tcgen05 contractions with f16 operands, float32 accumulate (bf16 tensors only) */
+    FAEDKV_DECODE_UMMA = 2,  /* tcgen05 contractions with f16 operands, float32 accumulate (bf16 tensors only) */
+    FAEDKV_DECODE_FFT = 3    /* float32 two-pass shared-memory FFTs (power-of-two P only): O(P log P) per
+                                query head instead of O(P * M)                                 */
 } faedkv_decode_mode;
 
 typedef struct {
@@ -163,6 +166,16 @@ int faedkv_reconstruct(faedkv_ctx *ctx, int layer, const float *coefK, const flo
 int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *coefK,
                        const float *coefV, const int32_t *t_len, int batch, float scale,
                        void *out, void *stream);
+
+/* IWDFT update and decode attention of one step in one call: exactly
+ * faedkv_append() followed by faedkv_decode_attn() (the new token is visible
+ * to the attention), but the update rides on the two passes that attention
+ * makes over the coefficient planes anyway, so the planes are read once and
+ * written once per step instead of read twice more.  coefK, coefV and t_len
+ * are updated in place; results equal those of the two separate calls. */
+int faedkv_append_decode_attn(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new,
+                              const void *q, int batch, float *coefK, float *coefV, int32_t *t_len,
+                              float scale, void *out, void *stream);
 
 /* Device-side status word of the context (host read; synchronises `stream`):
  * 0, or a nonzero code left by a kernel whose bounded wait on an mbarrier gave

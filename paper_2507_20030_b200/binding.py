@@ -21,13 +21,13 @@ LIB_PATH = os.path.join(_HERE, "lib", "libfaedkv.so")
 
 F32, BF16 = 0, 1
 PREFILL_AUTO, PREFILL_SIMT, PREFILL_UMMA = 0, 1, 2
-DECODE_AUTO, DECODE_SIMT, DECODE_UMMA = 0, 1, 2
+DECODE_AUTO, DECODE_SIMT, DECODE_UMMA, DECODE_FFT = 0, 1, 2, 3
 
 EXPORTS = [
     "faedkv_create", "faedkv_destroy", "faedkv_last_error", "faedkv_plan", "faedkv_n_bins",
     "faedkv_get_bins", "faedkv_coef_bytes", "faedkv_mask_lowpass", "faedkv_mask_mixed",
     "faedkv_compress_prefill", "faedkv_append", "faedkv_reconstruct", "faedkv_decode_attn",
-    "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
+    "faedkv_append_decode_attn", "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -86,6 +86,8 @@ def load() -> ctypes.CDLL:
     lib.faedkv_reconstruct.restype = _int
     lib.faedkv_decode_attn.argtypes = [_vp, _int, _vp, _vp, _vp, _vp, _int, ctypes.c_float, _vp, _vp]
     lib.faedkv_decode_attn.restype = _int
+    lib.faedkv_append_decode_attn.argtypes = [_vp, _int, _vp, _vp, _vp, _int, _vp, _vp, _vp, ctypes.c_float, _vp, _vp]
+    lib.faedkv_append_decode_attn.restype = _int
     lib.faedkv_device_status.argtypes = [_vp, _vp]
     lib.faedkv_device_status.restype = _int
     lib.faedkv_decode_attn_static.argtypes = [_int, _int, _int, _int, _vp, _int, _vp, _vp, _vp, _vp, _int,
@@ -243,6 +245,12 @@ class Context:
         self._check(self._lib.faedkv_decode_attn(
             self._h, layer, _ptr(q), _ptr(coefK), _ptr(coefV), _ptr(t_len), batch, float(scale),
             _ptr(out), _stream(stream)))
+
+    def append_decode_attn(self, layer, k_new, v_new, q, coefK, coefV, t_len, out, scale: float = 0.0, stream=None):
+        batch = q.shape[0]
+        self._check(self._lib.faedkv_append_decode_attn(
+            self._h, layer, _ptr(k_new), _ptr(v_new), _ptr(q), batch, _ptr(coefK), _ptr(coefV), _ptr(t_len),
+            float(scale), _ptr(out), _stream(stream)))
 
     def launch_count(self) -> int:
         return int(self._lib.faedkv_launch_count(self._h))

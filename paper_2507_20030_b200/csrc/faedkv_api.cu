@@ -15,6 +15,7 @@
 #include "k_prefill_umma.cuh"
 #include "k_idft_umma.cuh"
 #include "k_attn_umma.cuh"
+#include "k_attn_fft.cuh"
 
 using namespace faedkv;
 
@@ -25,6 +26,7 @@ struct LayerPlan {
     std::vector<int32_t> bins;
     int32_t *d_bins = nullptr;
     float *d_tab = nullptr;   // [M][16] per-bin phasors e^{jwk i}, i = 1..8 (tensor-core inverse transform)
+    int32_t *d_slot = nullptr;  // [P/2 + 1] bin -> index in bins[] or -1 (FFT-shaped transforms)
 };
 
 constexpr int kSplitsCap = 8;   // most position splits of the probability spectrum
@@ -34,6 +36,14 @@ struct TcScratch {
     __half *Qf16 = nullptr, *P16 = nullptr, *C16K = nullptr, *C16V = nullptr;
     float *S = nullptr, *tile_max = nullptr, *cmax = nullptr, *psum = nullptr, *colsum = nullptr, *PfS = nullptr;
     int gtot_max = 0, max_M = 0;
+};
+
+// Scratch of the FFT-shaped decode attention (power-of-two P).
+struct FftScratch {
+    float2 *Qs = nullptr, *Y = nullptr, *Zf = nullptr;
+    float *mloc = nullptr, *sloc = nullptr;
+    int max_M = 0;
+    bool attr_set = false;
 };
 
 }  // namespace
@@ -54,6 +64,8 @@ struct faedkv_ctx {
     UmmaPrefillState umma;             // tensor maps etc. of the tensor-core prefill
     TcScratch tc;
     bool use_tc = false;               // bf16 tensors and decode_mode != SIMT
+    bool use_fft = false;              // power-of-two P: FFT-shaped transforms in decode attention
+    FftScratch fs;
     unsigned long long launches = 0;   // kernels enqueued by this context so far
     std::string err;
 };
@@ -134,13 +146,17 @@ void free_scratch(faedkv_ctx *ctx) {
     cudaFree(t.Qf16); cudaFree(t.P16); cudaFree(t.C16K); cudaFree(t.C16V); cudaFree(t.S); cudaFree(t.tile_max);
     cudaFree(t.cmax); cudaFree(t.psum); cudaFree(t.colsum); cudaFree(t.PfS);
     t = TcScratch();
+    FftScratch &f = ctx->fs;
+    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc);
+    f = FftScratch();
 }
 
 // (Re)size the parts of the scratch area that depend on the largest M planned so far.
 int ensure_scratch(faedkv_ctx *ctx, int M) {
     const faedkv_config &c = ctx->cfg;
     const size_t B = (size_t)c.max_batch, P = (size_t)c.n_dft, HQP = (size_t)ctx->hqp;
-    if (ctx->S == nullptr) {
+    const bool attn_simt = !ctx->use_fft && !ctx->use_tc, attn_tc = !ctx->use_fft && ctx->use_tc;
+    if (attn_simt && ctx->S == nullptr) {
         const size_t n_tiles = (P + kTilePos - 1) / kTilePos;
         CUDA_TRY(ctx, cudaMalloc(&ctx->S, B * P * HQP * sizeof(float)));
         CUDA_TRY(ctx, cudaMalloc(&ctx->tile_max, B * n_tiles * HQP * sizeof(float)));
@@ -149,8 +165,10 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
     if (M > ctx->max_M) {
         cudaFree(ctx->Qf); cudaFree(ctx->Pf); cudaFree(ctx->partial);
         ctx->Qf = ctx->Pf = ctx->partial = nullptr;
-        CUDA_TRY(ctx, cudaMalloc(&ctx->Qf, B * 2 * (size_t)M * HQP * sizeof(float)));
-        CUDA_TRY(ctx, cudaMalloc(&ctx->Pf, B * 2 * (size_t)M * HQP * sizeof(float)));
+        if (attn_simt) {
+            CUDA_TRY(ctx, cudaMalloc(&ctx->Qf, B * 2 * (size_t)M * HQP * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&ctx->Pf, B * 2 * (size_t)M * HQP * sizeof(float)));
+        }
         // the slice count never exceeds 2*148 (units >= 1), nor ceil(M/64)
         int cap = (M + 63) / 64;
         if (cap > 2 * 148) cap = 2 * 148;
@@ -158,9 +176,25 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
         CUDA_TRY(ctx, cudaMalloc(&ctx->partial, B * c.n_kv_heads * (size_t)cap * ctx->gq * kHeadDim * sizeof(float)));
         ctx->max_M = M;
     }
+    if (ctx->use_fft) {
+        FftScratch &f = ctx->fs;
+        const fft::Geometry g = fft::make_geometry(c.n_dft, c.max_batch * c.n_q_heads);
+        if (f.Y == nullptr) {
+            CUDA_TRY(ctx, cudaMalloc(&f.Y, (size_t)g.N * g.Gp * sizeof(float2)));
+            CUDA_TRY(ctx, cudaMalloc(&f.Zf, (size_t)g.N * g.Gp * sizeof(float2)));
+            CUDA_TRY(ctx, cudaMalloc(&f.mloc, (size_t)g.N1 * g.Gp * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&f.sloc, (size_t)g.N1 * g.Gp * sizeof(float)));
+        }
+        if (M > f.max_M) {
+            cudaFree(f.Qs);
+            f.Qs = nullptr;
+            CUDA_TRY(ctx, cudaMalloc(&f.Qs, (size_t)M * g.Gp * sizeof(float2)));
+            f.max_M = M;
+        }
+    }
     if (ctx->use_tc) {
         TcScratch &t = ctx->tc;
-        if (t.S == nullptr) {
+        if (attn_tc && t.S == nullptr) {
             t.gtot_max = (c.max_batch * c.n_q_heads + 63) / 64 * 64;
             const size_t G = (size_t)t.gtot_max;
             CUDA_TRY(ctx, cudaMalloc(&t.S, P * G * sizeof(float)));
@@ -171,12 +205,14 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             CUDA_TRY(ctx, cudaMalloc(&t.P16, P * G * sizeof(__half)));
         }
         if (M > t.max_M) {
-            const size_t G = (size_t)t.gtot_max;
             cudaFree(t.Qf16); cudaFree(t.PfS); cudaFree(t.C16K); cudaFree(t.C16V);
             t.Qf16 = nullptr; t.PfS = nullptr; t.C16K = t.C16V = nullptr;
-            CUDA_TRY(ctx, cudaMalloc(&t.Qf16, 2 * (size_t)M * G * sizeof(__half)));
-            CUDA_TRY(ctx, cudaMemset(t.Qf16, 0, 2 * (size_t)M * G * sizeof(__half)));   // padded columns stay finite
-            CUDA_TRY(ctx, cudaMalloc(&t.PfS, (size_t)kSplitsCap * 2 * M * G * sizeof(float)));
+            if (attn_tc) {
+                const size_t G = (size_t)t.gtot_max;
+                CUDA_TRY(ctx, cudaMalloc(&t.Qf16, 2 * (size_t)M * G * sizeof(__half)));
+                CUDA_TRY(ctx, cudaMemset(t.Qf16, 0, 2 * (size_t)M * G * sizeof(__half)));   // padded columns stay finite
+                CUDA_TRY(ctx, cudaMalloc(&t.PfS, (size_t)kSplitsCap * 2 * M * G * sizeof(float)));
+            }
             const size_t cbytes = B * c.n_kv_heads * 2 * (size_t)M * kHeadDim * sizeof(__half);
             CUDA_TRY(ctx, cudaMalloc(&t.C16K, cbytes));
             CUDA_TRY(ctx, cudaMalloc(&t.C16V, cbytes));
@@ -340,6 +376,76 @@ int launch_attn_tc(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const flo
     return FAEDKV_OK;
 }
 
+// FFT-shaped decode attention; with APPEND the IWDFT update of K and V rides on the two coefficient
+// streams and the token counters advance at the end.
+template <typename TQ, int GQ, bool APPEND>
+int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const void *k_new, const void *v_new,
+                    float *coefK, float *coefV, int32_t *t_len, int batch, float scale, void *out, cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    FftScratch &f = ctx->fs;
+    const int H = c.n_kv_heads, HQ = c.n_q_heads, M = p.M, P = c.n_dft;
+    const fft::Geometry g = fft::make_geometry(P, batch * HQ);
+    const int col_blocks = g.Gp / fft::kCW;
+    const int kt = fft::transforms_per_cta(g.N1, g.N2, col_blocks);
+    const int mt = fft::transforms_per_cta(g.N2, g.N1, col_blocks);
+    const int lgKT = fft::ilog2(kt), lgMT = fft::ilog2(mt);
+    if (!f.attr_set) {
+        const uint32_t cap = (uint32_t)fft::smem_bytes(fft::kTileMax / fft::kCW, 1);
+        if (int r = opt_in_smem(ctx, k_afft_inv_a, cap)) return r;
+        if (int r = opt_in_smem(ctx, k_afft_mid, cap)) return r;
+        if (int r = opt_in_smem(ctx, k_afft_fwd_b, cap)) return r;
+        f.attr_set = true;
+    }
+    constexpr int KB = 16 / GQ;
+    {
+        dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
+        k_attn_qs<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(static_cast<const TQ *>(q), coefK,
+                                                                     static_cast<const TQ *>(k_new), t_len, p.d_bins, f.Qs, M, H,
+                                                                     HQ, g.Gp, (uint32_t)P, scale / (float)P);
+        if (int r = launch_check(ctx, "k_attn_qs")) return r;
+    }
+    {
+        dim3 grid(g.N2 >> lgKT, col_blocks);
+        k_afft_inv_a<<<grid, fft::kThreads, fft::smem_bytes(g.N1, kt), st>>>(g, p.d_slot, f.Qs, f.Y, lgKT);
+        if (int r = launch_check(ctx, "k_afft_inv_a")) return r;
+    }
+    {
+        dim3 grid(g.N1 >> lgMT, col_blocks);
+        k_afft_mid<<<grid, fft::kThreads, fft::smem_bytes(g.N2, mt), st>>>(g, f.Y, t_len, HQ, APPEND ? 1 : 0, f.mloc, f.sloc, lgMT);
+        if (int r = launch_check(ctx, "k_afft_mid")) return r;
+    }
+    {
+        dim3 grid(g.N2 >> lgKT, col_blocks);
+        k_afft_fwd_b<<<grid, fft::kThreads, fft::smem_bytes(g.N1, kt), st>>>(g, f.Y, f.mloc, lgMT, f.Zf, lgKT);
+        if (int r = launch_check(ctx, "k_afft_fwd_b")) return r;
+    }
+    {
+        const int slices = out_slices(ctx, batch, M);
+        const int per = (M + slices - 1) / slices;
+        dim3 grid(slices, batch * H);
+        k_attn_out_fft<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(coefV, static_cast<const TQ *>(v_new), t_len, f.Zf,
+                                                                          p.d_bins, ctx->partial, M, H, HQ, g, per);
+        if (int r = launch_check(ctx, "k_attn_out_fft")) return r;
+        k_attn_out_reduce_fft<TQ><<<batch * H * GQ, kHeadDim, 0, st>>>(ctx->partial, f.mloc, f.sloc, g.N1 >> lgMT, g.Gp,
+                                                                       static_cast<TQ *>(out), slices, GQ, 1.0f / (float)P,
+                                                                       t_len, APPEND ? batch : 0);
+        if (int r = launch_check(ctx, "k_attn_out_reduce_fft")) return r;
+    }
+    return FAEDKV_OK;
+}
+
+template <typename TQ, bool APPEND>
+int dispatch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const void *k_new, const void *v_new,
+                      float *coefK, float *coefV, int32_t *t_len, int batch, float scale, void *out, cudaStream_t st) {
+    switch (ctx->gq) {
+        case 1: return launch_attn_fft<TQ, 1, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
+        case 2: return launch_attn_fft<TQ, 2, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
+        case 4: return launch_attn_fft<TQ, 4, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
+        case 8: return launch_attn_fft<TQ, 8, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
+    }
+    return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be 1, 2, 4 or 8");
+}
+
 __global__ void k_set_tlen(int32_t *t_len, int batch, int T) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < batch) t_len[i] = T;
@@ -440,6 +546,9 @@ template <typename TQ>
 int dispatch_attn(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const float *coefK,
                   const float *coefV, const int32_t *t_len, int batch, float scale, void *out,
                   cudaStream_t st) {
+    if (ctx->use_fft)
+        return dispatch_attn_fft<TQ, false>(ctx, p, q, nullptr, nullptr, const_cast<float *>(coefK), const_cast<float *>(coefV),
+                                            const_cast<int32_t *>(t_len), batch, scale, out, st);
     if (ctx->use_tc) {
         switch (ctx->gq) {
             case 1: return launch_attn_tc<TQ, 1>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
@@ -471,8 +580,9 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     if (cfg->kv_dtype != FAEDKV_F32 && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->prefill_mode < FAEDKV_PREFILL_AUTO || cfg->prefill_mode > FAEDKV_PREFILL_UMMA) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->twiddle_terms < 0 || cfg->twiddle_terms > 2) return FAEDKV_ERR_INVALID_ARG;
-    if (cfg->decode_mode < FAEDKV_DECODE_AUTO || cfg->decode_mode > FAEDKV_DECODE_UMMA) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->decode_mode < FAEDKV_DECODE_AUTO || cfg->decode_mode > FAEDKV_DECODE_FFT) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->decode_mode == FAEDKV_DECODE_UMMA && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_UNSUPPORTED;
+    if (cfg->decode_mode == FAEDKV_DECODE_FFT && !fft::supported(cfg->n_dft)) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->head_dim != kHeadDim) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FAEDKV_ERR_UNSUPPORTED;
     const int gq = cfg->n_q_heads / cfg->n_kv_heads;
@@ -485,6 +595,8 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     ctx->gq = gq;
     ctx->hqp = (cfg->n_q_heads + 31) / 32 * 32;
     ctx->use_tc = cfg->kv_dtype == FAEDKV_BF16 && cfg->decode_mode != FAEDKV_DECODE_SIMT;
+    ctx->use_fft = fft::supported(cfg->n_dft) &&
+                   (cfg->decode_mode == FAEDKV_DECODE_AUTO || cfg->decode_mode == FAEDKV_DECODE_FFT);
     ctx->plans.resize(cfg->n_layers);
     if (cudaGetDevice(&ctx->device) != cudaSuccess ||
         cudaMalloc(&ctx->tick, sizeof(unsigned int) * (cfg->n_layers + 1)) != cudaSuccess ||
@@ -500,7 +612,7 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
 
 void faedkv_destroy(faedkv_ctx *ctx) {
     if (ctx == nullptr) return;
-    for (LayerPlan &p : ctx->plans) { cudaFree(p.d_bins); cudaFree(p.d_tab); }
+    for (LayerPlan &p : ctx->plans) { cudaFree(p.d_bins); cudaFree(p.d_tab); cudaFree(p.d_slot); }
     free_scratch(ctx);
     cudaFree(ctx->tick);
     delete ctx;
@@ -543,10 +655,23 @@ int faedkv_plan(faedkv_ctx *ctx, int layer, const uint8_t *bin_mask, int *n_bins
             return fail(ctx, FAEDKV_ERR_CUDA, "building the phasor table failed: %s", cudaGetErrorString(e));
         }
     }
+    int32_t *slot = nullptr;
+    if (ctx->use_fft) {
+        std::vector<int32_t> hs(n1, -1);
+        for (size_t i = 0; i < bins.size(); ++i) hs[bins[i]] = (int32_t)i;
+        e = cudaMalloc(&slot, (size_t)n1 * sizeof(int32_t));
+        if (e == cudaSuccess) e = cudaMemcpy(slot, hs.data(), (size_t)n1 * sizeof(int32_t), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            cudaFree(d); cudaFree(tab); cudaFree(slot);
+            return fail(ctx, FAEDKV_ERR_CUDA, "upload of the bin slot map failed: %s", cudaGetErrorString(e));
+        }
+    }
     cudaFree(p.d_bins);
     cudaFree(p.d_tab);
+    cudaFree(p.d_slot);
     p.d_bins = d;
     p.d_tab = tab;
+    p.d_slot = slot;
     p.M = (int)bins.size();
     p.bins.swap(bins);
     if (n_bins_out != nullptr) *n_bins_out = p.M;
@@ -692,6 +817,29 @@ int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *c
     if (ctx->cfg.kv_dtype == FAEDKV_BF16)
         return dispatch_attn<__nv_bfloat16>(ctx, *p, q, coefK, coefV, t_len, batch, scale, out, st);
     return dispatch_attn<float>(ctx, *p, q, coefK, coefV, t_len, batch, scale, out, st);
+}
+
+int faedkv_append_decode_attn(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new, const void *q,
+                              int batch, float *coefK, float *coefV, int32_t *t_len, float scale, void *out,
+                              void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    if (k_new == nullptr || v_new == nullptr || q == nullptr || coefK == nullptr || coefV == nullptr ||
+        t_len == nullptr || out == nullptr)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_append_decode_attn");
+    if (!(scale >= 0.0f)) return fail(ctx, FAEDKV_ERR_INVALID_ARG, "scale must be >= 0");
+    if (int r = check_ptrs(ctx, {k_new, v_new, q, coefK, coefV, out})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    if (!ctx->use_fft) {
+        if (int r = faedkv_append(ctx, layer, k_new, v_new, batch, coefK, coefV, t_len, stream)) return r;
+        return faedkv_decode_attn(ctx, layer, q, coefK, coefV, t_len, batch, scale, out, stream);
+    }
+    if (scale == 0.0f) scale = 1.0f / sqrtf((float)ctx->cfg.head_dim);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->cfg.kv_dtype == FAEDKV_BF16)
+        return dispatch_attn_fft<__nv_bfloat16, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
+    return dispatch_attn_fft<float, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
 }
 
 unsigned long long faedkv_launch_count(const faedkv_ctx *ctx) { return ctx ? ctx->launches : 0ULL; }

@@ -258,46 +258,129 @@ def test_all_bins_round_trip(fk):
 
 
 # ----------------------------------------------------------------------------- decode attention
+def _decode_modes(fk, dtype, P):
+    """Every evaluation of the two transforms that exists for this storage type and grid size."""
+    modes = [fk.DECODE_AUTO, fk.DECODE_SIMT]
+    if dtype == torch.bfloat16:
+        modes.append(fk.DECODE_UMMA)
+    if P & (P - 1) == 0 and P >= 64:
+        modes.append(fk.DECODE_FFT)
+    return modes
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("P,T,M,B,H,HQ,tl", [
-    (256, 256, 32, 2, 2, 8, None),        # GQA 4, full length
-    (200, 130, 37, 1, 3, 3, None),        # MHA (1 query head per kv head), t < P, odd sizes
-    (128, 128, 16, 2, 1, 8, [128, 70]),   # GQA 8, ragged lengths
-    (512, 512, 64, 1, 8, 32, None),       # 32 query heads, GQA 4
-    (128, 128, 24, 1, 20, 40, None),      # 40 query heads: two column blocks, GQA 2
+@pytest.mark.parametrize("P,T,M,B,H,HQ,tl,vscale", [
+    (256, 256, 32, 2, 2, 8, None, 1.0),        # GQA 4, full length
+    (200, 130, 37, 1, 3, 3, None, 1.0),        # MHA (1 query head per kv head), t < P, odd sizes
+    (128, 128, 16, 2, 1, 8, [128, 70], 1.0),   # GQA 8, ragged lengths
+    (512, 512, 64, 1, 8, 32, None, 1.0),       # 32 query heads, GQA 4
+    (128, 128, 24, 1, 20, 40, None, 1.0),      # 40 query heads: two column blocks, GQA 2
+    # smallest FFT-shaped grid, every bin retained, odd live length.  With all bins and few tokens the
+    # softmax is sharp and the output is close to single rows of V; V is scaled so that the bf16 output
+    # grid (relative 2^-9) stays finer than the absolute tolerance.
+    (64, 64, 33, 1, 2, 4, [33], 0.125),
+    (4096, 4096, 96, 3, 2, 8, [4096, 1, 2049], 0.125),   # two-pass split 64 x 32; a one-token sequence
 ])
-def test_decode_attn_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, tl):
+def test_decode_attn_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, tl, vscale):
     from paper_2507_20030_b200 import synth
-    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
-                     prefill_mode=fk.PREFILL_SIMT)
     mask = _random_mask(P, M, 3 * P + M)
+    mask[0] = 1
+    M = int(mask.sum())
+    bins = oracle.plan(P, mask)
+    K, V = _make(21 + P, B, H, T, dtype)
+    V = (V * vscale).to(dtype)                # a power of two: exact in either storage type
+    q = synth.make_q(5, 0, B, HQ, 128, dtype=dtype)
+    want = want2 = None
+    for mode in _decode_modes(fk, dtype, P):
+        ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                         prefill_mode=fk.PREFILL_SIMT, decode_mode=mode)
+        ctx.plan(0, mask)
+        cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+        t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+        ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+        if tl is not None:
+            # shorter sequences: recompute their state from the first tl[b] tokens only
+            for b, t in enumerate(tl):
+                if t < T:
+                    Kb, Vb = K[b:b + 1, :, :t].contiguous().cuda(), V[b:b + 1, :, :t].contiguous().cuda()
+                    ctx.compress_prefill(0, Kb, Vb, cK[b:b + 1], cV[b:b + 1], t_len[b:b + 1])
+        out = torch.full((B, HQ, 128), float("nan"), dtype=dtype, device="cuda")
+        ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out)
+        torch.cuda.synchronize()
+        t_np = t_len.cpu().numpy()
+        if want is None:
+            want = oracle_decode_attn(oracle, q, to_np64(cK), to_np64(cV), P, bins, t_np)
+            want2 = oracle_decode_attn(oracle, q, to_np64(cK), to_np64(cV), P, bins, t_np, scale=0.05)
+        err = np.abs(to_np64(out) - want).max()
+        assert err <= ATTN_MAX_ABS, (mode, err)
+        # explicit scale
+        out2 = torch.empty_like(out)
+        ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out2, scale=0.05)
+        torch.cuda.synchronize()
+        err2 = np.abs(to_np64(out2) - want2).max()
+        assert err2 <= ATTN_MAX_ABS, (mode, err2)
+        assert ctx.device_status() == 0
+        ctx.close()
+
+
+@pytest.mark.parametrize("P,M,B,H,HQ", [(32768, 48, 1, 2, 8), (131072, 32, 2, 1, 4), (16384, 64, 3, 2, 4)])
+def test_decode_attn_fft_long_grids(fk, oracle, P, M, B, H, HQ):
+    """FFT-shaped transforms at the grid sizes of the long-context workloads (few bins, so that the
+    oracle's materialised reconstruction stays cheap); ragged live lengths."""
+    from paper_2507_20030_b200 import synth
+    dtype = torch.bfloat16
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=fk.BF16,
+                     decode_mode=fk.DECODE_FFT)
+    mask = fk.mask_mixed(P, M, 3, 17)
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    rng = np.random.default_rng(P + M)
+    amp = np.sqrt(P) * np.exp(-np.arange(M) / (M / 3.0))[None, None, None, :, None]
+    cK = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * amp).astype(np.float32)).cuda()
+    cV = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * amp).astype(np.float32)).cuda()
+    t_np = np.array([P, P // 3 + 1, 5][:B], dtype=np.int32)
+    t_len = torch.from_numpy(t_np).cuda()
+    q = synth.make_q(9, 1, B, HQ, 128, dtype=dtype)
+    out = torch.empty((B, HQ, 128), dtype=dtype, device="cuda")
+    ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out)
+    torch.cuda.synchronize()
+    want = oracle_decode_attn(oracle, q, to_np64(cK), to_np64(cV), P, bins, t_np)
+    err = np.abs(to_np64(out) - want).max()
+    assert err <= ATTN_MAX_ABS, err
+    ctx.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,M,B,H,HQ,t0", [(256, 40, 2, 2, 8, [100, 255]), (1024, 65, 1, 3, 6, [3000]),
+                                           (200, 30, 2, 1, 2, [7, 199])])
+def test_append_decode_attn_equals_the_two_calls(fk, oracle, dtype, P, M, B, H, HQ, t0):
+    """The fused step: planes and counters bit-identical to faedkv_append, output equal to the oracle's
+    attention on the updated state."""
+    from paper_2507_20030_b200 import synth
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype))
+    mask = _random_mask(P, M, P + 3 * M)
     mask[0] = 1
     M = int(mask.sum())
     ctx.plan(0, mask)
     bins = oracle.plan(P, mask)
-    K, V = _make(21 + P, B, H, T, dtype)
-    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
-    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
-    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
-    if tl is not None:
-        # shorter sequences: recompute their state from the first tl[b] tokens only
-        for b, t in enumerate(tl):
-            if t < T:
-                Kb, Vb = K[b:b + 1, :, :t].contiguous().cuda(), V[b:b + 1, :, :t].contiguous().cuda()
-                ctx.compress_prefill(0, Kb, Vb, cK[b:b + 1], cV[b:b + 1], t_len[b:b + 1])
-    q = synth.make_q(5, 0, B, HQ, 128, dtype=dtype)
+    rng = np.random.default_rng(M)
+    cK = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * 4).astype(np.float32)).cuda()
+    cV = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * 4).astype(np.float32)).cuda()
+    sK, sV = cK.clone(), cV.clone()
+    t_np = np.array(t0, dtype=np.int32)
+    t_len = torch.from_numpy(t_np.copy()).cuda()
+    t_sep = t_len.clone()
     out = torch.empty((B, HQ, 128), dtype=dtype, device="cuda")
-    ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out)
-    torch.cuda.synchronize()
-    t_np = t_len.cpu().numpy()
-    want = oracle_decode_attn(oracle, q, to_np64(cK), to_np64(cV), P, bins, t_np)
-    assert np.abs(to_np64(out) - want).max() <= ATTN_MAX_ABS
-    # explicit scale
-    out2 = torch.empty_like(out)
-    ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out2, scale=0.05)
-    torch.cuda.synchronize()
-    want2 = oracle_decode_attn(oracle, q, to_np64(cK), to_np64(cV), P, bins, t_np, scale=0.05)
-    assert np.abs(to_np64(out2) - want2).max() <= ATTN_MAX_ABS
+    for s in range(3):
+        k, v = synth.make_token(31, s, B, H, 128, pos=int(t_np[0]) + s, dtype=dtype)
+        q = synth.make_q(31, s, B, HQ, 128, dtype=dtype)
+        ctx.append_decode_attn(0, k.cuda(), v.cuda(), q.cuda(), cK, cV, t_len, out)
+        ctx.append(0, k.cuda(), v.cuda(), sK, sV, t_sep)
+        torch.cuda.synchronize()
+        assert torch.equal(cK, sK) and torch.equal(cV, sV) and torch.equal(t_len, t_sep)
+        want = oracle_decode_attn(oracle, q, to_np64(sK), to_np64(sV), P, bins, t_np + s + 1)
+        err = np.abs(to_np64(out) - want).max()
+        assert err <= ATTN_MAX_ABS, (s, err)
     ctx.close()
 
 
