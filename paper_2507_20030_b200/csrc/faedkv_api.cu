@@ -41,9 +41,10 @@ struct TcScratch {
 // Scratch of the FFT-shaped decode attention (power-of-two P).
 struct FftScratch {
     float2 *Qs = nullptr, *Y = nullptr, *Zf = nullptr;
-    float *mloc = nullptr, *sloc = nullptr;
+    float *mloc = nullptr, *sloc = nullptr, *colsum = nullptr;
+    unsigned int *tickets = nullptr;      // [max_batch * H + max_batch], zero between calls
     int max_M = 0;
-    bool attr_set = false;
+    unsigned int attr_mask[3] = {0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
 };
 
 }  // namespace
@@ -147,7 +148,7 @@ void free_scratch(faedkv_ctx *ctx) {
     cudaFree(t.cmax); cudaFree(t.psum); cudaFree(t.colsum); cudaFree(t.PfS);
     t = TcScratch();
     FftScratch &f = ctx->fs;
-    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc);
+    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.tickets);
     f = FftScratch();
 }
 
@@ -184,6 +185,10 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             CUDA_TRY(ctx, cudaMalloc(&f.Zf, (size_t)g.N * g.Gp * sizeof(float2)));
             CUDA_TRY(ctx, cudaMalloc(&f.mloc, (size_t)g.N1 * g.Gp * sizeof(float)));
             CUDA_TRY(ctx, cudaMalloc(&f.sloc, (size_t)g.N1 * g.Gp * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&f.colsum, (size_t)g.Gp * sizeof(float)));
+            const size_t n_tickets = (size_t)c.max_batch * c.n_kv_heads + c.max_batch;
+            CUDA_TRY(ctx, cudaMalloc(&f.tickets, n_tickets * sizeof(unsigned int)));
+            CUDA_TRY(ctx, cudaMemset(f.tickets, 0, n_tickets * sizeof(unsigned int)));
         }
         if (M > f.max_M) {
             cudaFree(f.Qs);
@@ -376,6 +381,28 @@ int launch_attn_tc(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const flo
     return FAEDKV_OK;
 }
 
+// Launch one of the three FFT kernels for a transform length of 2^lg rows.
+#define FAEDKV_FFT_SWITCH(lg, lo, CALL)                                                     \
+    switch (lg) {                                                                           \
+        case 2: if (lo <= 2) { CALL(2); } break;                                            \
+        case 3: CALL(3); break;                                                             \
+        case 4: CALL(4); break;                                                             \
+        case 5: CALL(5); break;                                                             \
+        case 6: CALL(6); break;                                                             \
+        case 7: CALL(7); break;                                                             \
+        case 8: CALL(8); break;                                                             \
+        case 9: CALL(9); break;                                                             \
+        default: break;                                                                     \
+    }
+
+template <typename K>
+int fft_opt_in(faedkv_ctx *ctx, K kernel, size_t bytes, unsigned int &done_mask, int lg) {
+    if (bytes <= 48 * 1024 || (done_mask >> lg) & 1u) return FAEDKV_OK;
+    if (int r = opt_in_smem(ctx, kernel, (uint32_t)bytes)) return r;
+    done_mask |= 1u << lg;
+    return FAEDKV_OK;
+}
+
 // FFT-shaped decode attention; with APPEND the IWDFT update of K and V rides on the two coefficient
 // streams and the token counters advance at the end.
 template <typename TQ, int GQ, bool APPEND>
@@ -386,16 +413,8 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
     const int H = c.n_kv_heads, HQ = c.n_q_heads, M = p.M, P = c.n_dft;
     const fft::Geometry g = fft::make_geometry(P, batch * HQ);
     const int col_blocks = g.Gp / fft::kCW;
-    const int kt = fft::transforms_per_cta(g.N1, g.N2, col_blocks);
-    const int mt = fft::transforms_per_cta(g.N2, g.N1, col_blocks);
-    const int lgKT = fft::ilog2(kt), lgMT = fft::ilog2(mt);
-    if (!f.attr_set) {
-        const uint32_t cap = (uint32_t)fft::smem_bytes(fft::kTileMax / fft::kCW, 1);
-        if (int r = opt_in_smem(ctx, k_afft_inv_a, cap)) return r;
-        if (int r = opt_in_smem(ctx, k_afft_mid, cap)) return r;
-        if (int r = opt_in_smem(ctx, k_afft_fwd_b, cap)) return r;
-        f.attr_set = true;
-    }
+    const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks));
+    const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks));
     constexpr int KB = 16 / GQ;
     {
         dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
@@ -404,32 +423,50 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
                                                                      HQ, g.Gp, (uint32_t)P, scale / (float)P);
         if (int r = launch_check(ctx, "k_attn_qs")) return r;
     }
+    int rc = FAEDKV_ERR_UNSUPPORTED;
     {
-        dim3 grid(g.N2 >> lgKT, col_blocks);
-        k_afft_inv_a<<<grid, fft::kThreads, fft::smem_bytes(g.N1, kt), st>>>(g, p.d_slot, f.Qs, f.Y, lgKT);
+        const dim3 grid(g.N2 >> lgKT, col_blocks);
+        const size_t smem = afft_smem_a(g.lgN1, lgKT, true);
+#define CALL(LG)                                                                                         \
+        rc = fft_opt_in(ctx, k_afft_inv_a<LG>, smem, f.attr_mask[0], LG);                                \
+        if (rc == 0) k_afft_inv_a<LG><<<grid, fft::kThreads, smem, st>>>(g, p.d_slot, f.Qs, f.Y, lgKT)
+        FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
+#undef CALL
+        if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
         if (int r = launch_check(ctx, "k_afft_inv_a")) return r;
     }
+    rc = FAEDKV_ERR_UNSUPPORTED;
     {
-        dim3 grid(g.N1 >> lgMT, col_blocks);
-        k_afft_mid<<<grid, fft::kThreads, fft::smem_bytes(g.N2, mt), st>>>(g, f.Y, t_len, HQ, APPEND ? 1 : 0, f.mloc, f.sloc, lgMT);
+        const dim3 grid(g.N1 >> lgMT, col_blocks);
+        const size_t smem = afft_smem_mid(g.lgN2, lgMT);
+#define CALL(LG)                                                                                         \
+        rc = fft_opt_in(ctx, k_afft_mid<LG>, smem, f.attr_mask[1], LG);                                  \
+        if (rc == 0) k_afft_mid<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Y, t_len, HQ, APPEND ? 1 : 0, f.mloc, f.sloc, lgMT)
+        FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
+#undef CALL
+        if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
         if (int r = launch_check(ctx, "k_afft_mid")) return r;
     }
+    rc = FAEDKV_ERR_UNSUPPORTED;
     {
-        dim3 grid(g.N2 >> lgKT, col_blocks);
-        k_afft_fwd_b<<<grid, fft::kThreads, fft::smem_bytes(g.N1, kt), st>>>(g, f.Y, f.mloc, lgMT, f.Zf, lgKT);
+        const dim3 grid(g.N2 >> lgKT, col_blocks);
+        const size_t smem = afft_smem_fwd_b(g.lgN1, lgKT, lgMT);
+#define CALL(LG)                                                                                         \
+        rc = fft_opt_in(ctx, k_afft_fwd_b<LG>, smem, f.attr_mask[2], LG);                                \
+        if (rc == 0) k_afft_fwd_b<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Y, f.mloc, f.sloc, lgMT, f.Zf, f.colsum, lgKT)
+        FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
+#undef CALL
+        if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
         if (int r = launch_check(ctx, "k_afft_fwd_b")) return r;
     }
     {
         const int slices = out_slices(ctx, batch, M);
         const int per = (M + slices - 1) / slices;
         dim3 grid(slices, batch * H);
-        k_attn_out_fft<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(coefV, static_cast<const TQ *>(v_new), t_len, f.Zf,
-                                                                          p.d_bins, ctx->partial, M, H, HQ, g, per);
+        k_attn_out_fft<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(
+            coefV, static_cast<const TQ *>(v_new), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
+            static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P);
         if (int r = launch_check(ctx, "k_attn_out_fft")) return r;
-        k_attn_out_reduce_fft<TQ><<<batch * H * GQ, kHeadDim, 0, st>>>(ctx->partial, f.mloc, f.sloc, g.N1 >> lgMT, g.Gp,
-                                                                       static_cast<TQ *>(out), slices, GQ, 1.0f / (float)P,
-                                                                       t_len, APPEND ? batch : 0);
-        if (int r = launch_check(ctx, "k_attn_out_reduce_fft")) return r;
     }
     return FAEDKV_OK;
 }

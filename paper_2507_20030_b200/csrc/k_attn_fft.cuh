@@ -8,8 +8,8 @@
 //   (3,4)                pass A' of the forward transform of p~, in place            -> Y
 //       k_afft_fwd_b     rescale every tile to the column's global maximum, pass B'  -> Zf
 //   (5) k_attn_out_fft   Pf at the retained bins from Zf (unpacking formula), out partials from one pass
-//                        over C_V (with APPEND the update of C_V on the way)
-//       k_attn_out_reduce_fft   sum partials, divide by P * (softmax normaliser); APPEND: t_len += 1
+//                        over C_V (with APPEND the update of C_V on the way); the last CTA of a kv head
+//                        sums the partials and divides by P * (softmax normaliser); APPEND: t_len += 1
 //
 // The scores never leave shared memory; the only intermediates in (L2-resident) global memory are the
 // two-pass arrays Y, Zf of P/2 complex values per column and the per-tile softmax statistics.
@@ -87,60 +87,75 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
 
 // ---- (2) pass A of the inverse transform, half-spectrum packing fused into the load ----------------
 // slot[k], k in [0, N]: index of one-sided bin k in the plan, or -1.  Y: [N1][N2][Gp].
-// grid = (N2 / KT, Gp / 16); block = 256; dynamic smem = fft::smem_bytes(N1, KT).
+// grid = (N2 / KT, Gp / 16); block = 256; dynamic smem = afft_smem_a(lgN1, lgKT, true).
+template <int LG>
 __global__ void __launch_bounds__(fft::kThreads)
 k_afft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float2 *__restrict__ Qs,
              float2 *__restrict__ Y, int lgKT) {
     using namespace fft;
+    constexpr int NF = 1 << LG;                      // = N1
     extern __shared__ float2 fft_smem[];
-    const int KT = 1 << lgKT, lg_cols = lgKT + 4;
-    const int tile = g.N1 << lg_cols;
-    float2 *a = fft_smem, *b = fft_smem + tile, *tw = fft_smem + 2 * tile;
-    fill_twiddles(tw, g.N1);
+    const int KT = 1 << lgKT, lg_cols = lgKT + kLgCW;
+    const int tile = NF << lg_cols;
+    float2 *xa = fft_smem, *xb = xa + (exchange_buffers(LG) > 0 ? tile : 0);
+    float2 *tw = xb + (exchange_buffers(LG) > 1 ? tile : 0);
+    float2 *tab_i = tw + NF;                         // [m1][kt]: e^{+j2pi k2 m1 / N}
+    float2 *tab_p = tab_i + (NF << lgKT);            // [k1][kt]: e^{+j2pi (N2 k1 + k2) / P}
     const int k2_0 = blockIdx.x * KT, g0 = blockIdx.y * kCW;
-    for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int c = e & (kCW - 1), kt = (e >> 4) & (KT - 1), k1 = e >> lg_cols;
+    fill_twiddles(tw, NF);
+    for (int e = threadIdx.x; e < (NF << lgKT); e += kThreads) {
+        const int kt = e & (KT - 1), r = e >> lgKT;
+        tab_i[e] = unit_phasor((uint32_t)((k2_0 + kt) * r), (uint32_t)g.N);      // k2 * m1 < N2 * N1 = N
+        tab_p[e] = unit_phasor((uint32_t)(g.N2 * r + k2_0 + kt), g.P);
+    }
+    __syncthreads();
+    auto load = [&](int k1, int cidx) {
+        const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
         const int k = g.N2 * k1 + k2_0 + kt;                 // 0 <= k < N
         const int col = g0 + c;
         float2 z = make_float2(0.f, 0.f);
-        if (col < g.G) {
-            const int sa = slot[k], sb = slot[g.N - k];
-            if (sa >= 0 || sb >= 0) {
-                const float2 xa = sa >= 0 ? Qs[(size_t)sa * g.Gp + col] : make_float2(0.f, 0.f);
-                float2 xb = sb >= 0 ? Qs[(size_t)sb * g.Gp + col] : make_float2(0.f, 0.f);
-                xb.y = -xb.y;                                            // conj X[N-k]
-                const float2 s = cadd(xa, xb), d = csub(xa, xb);
-                z = cadd(s, cmulj(cmul(unit_phasor((uint32_t)k, g.P), d)));
-            }
+        const int sa = slot[k], sb = slot[g.N - k];
+        if ((sa >= 0 || sb >= 0) && col < g.G) {
+            const float2 xk = sa >= 0 ? Qs[(size_t)sa * g.Gp + col] : make_float2(0.f, 0.f);
+            float2 xm = sb >= 0 ? Qs[(size_t)sb * g.Gp + col] : make_float2(0.f, 0.f);
+            xm.y = -xm.y;                                            // conj X[N-k]
+            z = cadd(cadd(xk, xm), cmulj(cmul(tab_p[(k1 << lgKT) + kt], csub(xk, xm))));
         }
-        a[e] = z;
-    }
-    __syncthreads();
-    const float2 *res = fft_tile(a, b, tw, g.N1, lg_cols);
-    for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int c = e & (kCW - 1), kt = (e >> 4) & (KT - 1), m1 = e >> lg_cols;
-        const int k2 = k2_0 + kt;
-        Y[y_index(g, m1, k2, g0 + c)] = cmul(res[e], unit_phasor((uint32_t)(k2 * m1), (uint32_t)g.N));
-    }
+        return z;
+    };
+    auto store = [&](int m1, int cidx, float2 v) {
+        const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
+        Y[y_index(g, m1, k2_0 + kt, g0 + c)] = cmul(v, tab_i[(m1 << lgKT) + kt]);
+    };
+    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
 }
 
 // ---- pass B of the inverse transform, local softmax, pass A' of the forward transform ---------------
 // One CTA = MT values of m1 (one "tile" of the softmax statistics) x 16 columns.
 // mloc, sloc: [N1 / MT][Gp].  live length of a column = min(t_len[col / HQ] + t_add, P).
-// grid = (N1 / MT, Gp / 16); block = 256; dynamic smem = fft::smem_bytes(N2, MT).
+// grid = (N1 / MT, Gp / 16); block = 256; dynamic smem = afft_smem_mid(lgN2, lgMT).
+template <int LG>
 __global__ void __launch_bounds__(fft::kThreads)
 k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ t_len, int HQ, int t_add,
            float *__restrict__ mloc, float *__restrict__ sloc, int lgMT) {
     using namespace fft;
+    constexpr int NF = 1 << LG;                      // = N2
     extern __shared__ float2 fft_smem[];
     __shared__ float red[kThreads];
     __shared__ float colv[kCW];
     __shared__ int live_s[kCW];
-    const int MT = 1 << lgMT, lg_cols = lgMT + 4;
-    const int tile = g.N2 << lg_cols;
-    float2 *a = fft_smem, *b = fft_smem + tile, *tw = fft_smem + 2 * tile;
-    fill_twiddles(tw, g.N2);
+    const int MT = 1 << lgMT, lg_cols = lgMT + kLgCW;
+    const int tile = NF << lg_cols;
+    float2 *T = fft_smem;                            // scores / probabilities of this tile
+    float2 *xa = T + tile, *xb = xa + (exchange_buffers(LG) > 0 ? tile : 0);
+    float2 *tw = xb + (exchange_buffers(LG) > 1 ? tile : 0);
+    float2 *tab_i = tw + NF;                         // [k1'][mt]: e^{+j2pi k1' m1 / N}
     const int m1_0 = blockIdx.x * MT, g0 = blockIdx.y * kCW;
+    fill_twiddles(tw, NF);
+    for (int e = threadIdx.x; e < (NF << lgMT); e += kThreads) {
+        const int mt = e & (MT - 1), r = e >> lgMT;
+        tab_i[e] = unit_phasor((uint32_t)((m1_0 + mt) * r), (uint32_t)g.N);
+    }
     if (threadIdx.x < kCW) {
         const int col = g0 + threadIdx.x;
         int live = 0;
@@ -150,20 +165,23 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
         }
         live_s[threadIdx.x] = live;
     }
-    for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int c = e & (kCW - 1), mt = (e >> 4) & (MT - 1), row = e >> lg_cols;
-        a[e] = Y[y_index(g, m1_0 + mt, row, g0 + c)];
+    __syncthreads();
+    {
+        auto load = [&](int k2, int cidx) {
+            return Y[y_index(g, m1_0 + (cidx >> kLgCW), k2, g0 + (cidx & (kCW - 1)))];
+        };
+        auto store = [&](int m2, int cidx, float2 v) { T[(m2 << lg_cols) + cidx] = v; };
+        fft_rows<LG>(lg_cols, xa, xb, tw, load, store);      // T[m2][mt, c] = z[m1 + N1 m2]
     }
     __syncthreads();
-    float2 *res = fft_tile(a, b, tw, g.N2, lg_cols);        // rows are now m2; element = z[m1 + N1 m2]
     // a thread always meets the same column: kThreads is a multiple of 16
     const int c = threadIdx.x & (kCW - 1);
     const int live = live_s[c];
     float mx = -INFINITY;
     for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int mt = (e >> 4) & (MT - 1), m2 = e >> lg_cols;
+        const int mt = (e >> kLgCW) & (MT - 1), m2 = e >> lg_cols;
         const int n0 = 2 * (m1_0 + mt + g.N1 * m2);
-        const float2 v = res[e];
+        const float2 v = T[e];
         if (n0 < live) mx = fmaxf(mx, v.x);
         if (n0 + 1 < live) mx = fmaxf(mx, v.y);
     }
@@ -179,13 +197,13 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
     const float mcol = colv[c];
     float sum = 0.f;
     for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int mt = (e >> 4) & (MT - 1), m2 = e >> lg_cols;
+        const int mt = (e >> kLgCW) & (MT - 1), m2 = e >> lg_cols;
         const int n0 = 2 * (m1_0 + mt + g.N1 * m2);
-        const float2 v = res[e];
+        const float2 v = T[e];
         const float pe = n0 < live ? __expf(v.x - mcol) : 0.f;
         const float po = n0 + 1 < live ? __expf(v.y - mcol) : 0.f;
         sum += pe + po;
-        res[e] = make_float2(pe, po);
+        T[e] = make_float2(pe, po);
     }
     red[threadIdx.x] = sum;
     __syncthreads();
@@ -196,35 +214,42 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
         mloc[(size_t)blockIdx.x * g.Gp + g0 + threadIdx.x] = colv[threadIdx.x];
         sloc[(size_t)blockIdx.x * g.Gp + g0 + threadIdx.x] = s;
     }
-    const float2 *res2 = fft_tile(res, res == a ? b : a, tw, g.N2, lg_cols);   // rows are now k1'
-    for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int cc = e & (kCW - 1), mt = (e >> 4) & (MT - 1), k1p = e >> lg_cols;
-        const int m1 = m1_0 + mt;
-        Y[y_index(g, m1, k1p, g0 + cc)] = cmul(res2[e], unit_phasor((uint32_t)(k1p * m1), (uint32_t)g.N));
+    {
+        auto load = [&](int m2, int cidx) { return T[(m2 << lg_cols) + cidx]; };
+        auto store = [&](int k1p, int cidx, float2 v) {
+            const int mt = cidx >> kLgCW;
+            Y[y_index(g, m1_0 + mt, k1p, g0 + (cidx & (kCW - 1)))] = cmul(v, tab_i[(k1p << lgMT) + mt]);
+        };
+        fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
     }
 }
 
 // ---- pass B' of the forward transform ---------------------------------------------------------------
 // Every softmax tile is first brought to the column's global maximum: factor exp(mloc - max_tiles mloc).
+// The CTAs with blockIdx.x == 0 also write the softmax normaliser colsum[col] = sum_tiles sloc * factor.
 // Zf: [N][Gp], index k1' + N2 * k2'.
-// grid = (N2 / KT, Gp / 16); block = 256; dynamic smem = fft::smem_bytes(N1, KT).
+// grid = (N2 / KT, Gp / 16); block = 256; dynamic smem = afft_smem_a(lgN1, lgKT, false) + factors.
+template <int LG>
 __global__ void __launch_bounds__(fft::kThreads)
-k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restrict__ mloc, int lgMT,
-             float2 *__restrict__ Zf, int lgKT) {
+k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restrict__ mloc,
+             const float *__restrict__ sloc, int lgMT, float2 *__restrict__ Zf, float *__restrict__ colsum, int lgKT) {
     using namespace fft;
+    constexpr int NF = 1 << LG;                      // = N1
     extern __shared__ float2 fft_smem[];
     __shared__ float red[kThreads];
     __shared__ float mg[kCW];
-    const int KT = 1 << lgKT, lg_cols = lgKT + 4;
-    const int tile = g.N1 << lg_cols;
-    float2 *a = fft_smem, *b = fft_smem + tile, *tw = fft_smem + 2 * tile;
-    fill_twiddles(tw, g.N1);
-    const int k1_0 = blockIdx.x * KT, g0 = blockIdx.y * kCW;
-    const int n_tiles = g.N1 >> lgMT;
+    const int lg_cols = lgKT + kLgCW;
+    const int tile = NF << lg_cols;
+    float2 *xa = fft_smem, *xb = xa + (exchange_buffers(LG) > 0 ? tile : 0);
+    float2 *tw = xb + (exchange_buffers(LG) > 1 ? tile : 0);
+    float *fac = reinterpret_cast<float *>(tw + NF);  // [n_tiles][16]
+    const int k1_0 = blockIdx.x << lgKT, g0 = blockIdx.y * kCW;
+    const int n_tiles = NF >> lgMT;
+    fill_twiddles(tw, NF);
+    const int c = threadIdx.x & (kCW - 1);
     {
-        const int c = threadIdx.x & (kCW - 1);
         float mx = -INFINITY;
-        for (int ti = threadIdx.x >> 4; ti < n_tiles; ti += kThreads / kCW) mx = fmaxf(mx, mloc[(size_t)ti * g.Gp + g0 + c]);
+        for (int ti = threadIdx.x >> kLgCW; ti < n_tiles; ti += kThreads / kCW) mx = fmaxf(mx, mloc[(size_t)ti * g.Gp + g0 + c]);
         red[threadIdx.x] = mx;
         __syncthreads();
         if (threadIdx.x < kCW) {
@@ -234,31 +259,77 @@ k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restr
             mg[threadIdx.x] = m;
         }
         __syncthreads();
+        const float m = mg[c];
+        float part = 0.f;
+        for (int ti = threadIdx.x >> kLgCW; ti < n_tiles; ti += kThreads / kCW) {
+            const float ml = mloc[(size_t)ti * g.Gp + g0 + c];
+            const float f = ml == -INFINITY ? 0.f : __expf(ml - m);
+            fac[ti * kCW + c] = f;
+            if (blockIdx.x == 0) part += f * sloc[(size_t)ti * g.Gp + g0 + c];
+        }
+        if (blockIdx.x == 0) {
+            __syncthreads();
+            red[threadIdx.x] = part;
+            __syncthreads();
+            if (threadIdx.x < kCW) {
+                float s = red[threadIdx.x];
+#pragma unroll
+                for (int i = 1; i < kThreads / kCW; ++i) s += red[threadIdx.x + kCW * i];
+                colsum[g0 + threadIdx.x] = s;
+            }
+        }
+        __syncthreads();
     }
-    for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int c = e & (kCW - 1), kt = (e >> 4) & (KT - 1), m1 = e >> lg_cols;
-        const float ml = mloc[(size_t)(m1 >> lgMT) * g.Gp + g0 + c];
-        const float f = ml == -INFINITY ? 0.f : __expf(ml - mg[c]);
-        const float2 v = U[y_index(g, m1, k1_0 + kt, g0 + c)];
-        a[e] = make_float2(v.x * f, v.y * f);
-    }
-    __syncthreads();
-    const float2 *res = fft_tile(a, b, tw, g.N1, lg_cols);   // rows are now k2'
-    for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int c = e & (kCW - 1), kt = (e >> 4) & (KT - 1), k2p = e >> lg_cols;
-        Zf[((size_t)(k1_0 + kt) + (size_t)g.N2 * k2p) * g.Gp + g0 + c] = res[e];
-    }
+    auto load = [&](int m1, int cidx) {
+        const int cc = cidx & (kCW - 1);
+        const float f = fac[(m1 >> lgMT) * kCW + cc];
+        const float2 v = U[y_index(g, m1, k1_0 + (cidx >> kLgCW), g0 + cc)];
+        return make_float2(v.x * f, v.y * f);
+    };
+    auto store = [&](int k2p, int cidx, float2 v) {
+        Zf[((size_t)(k1_0 + (cidx >> kLgCW)) + (size_t)g.N2 * k2p) * g.Gp + g0 + (cidx & (kCW - 1))] = v;
+    };
+    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+}
+
+// Dynamic shared memory of the three kernels above (bytes).
+inline size_t afft_smem_a(int lg, int lgKT, bool packing_table) {
+    const size_t nf = (size_t)1 << lg, tile = nf << (lgKT + fft::kLgCW);
+    return (fft::exchange_buffers(lg) * tile + nf + (packing_table ? 2 : 1) * (nf << lgKT)) * sizeof(float2);
+}
+inline size_t afft_smem_mid(int lg, int lgMT) {
+    const size_t nf = (size_t)1 << lg, tile = nf << (lgMT + fft::kLgCW);
+    return ((1 + fft::exchange_buffers(lg)) * tile + nf + (nf << lgMT)) * sizeof(float2);
+}
+inline size_t afft_smem_fwd_b(int lg, int lgKT, int lgMT) {
+    const size_t nf = (size_t)1 << lg, tile = nf << (lgKT + fft::kLgCW);
+    return (fft::exchange_buffers(lg) * tile + nf) * sizeof(float2) + ((nf >> lgMT) * fft::kCW) * sizeof(float);
 }
 
 // ---- (5) ------------------------------------------------------------------------------------------
+// One pass over C_V.  A CTA takes a slice of the bins of one (sequence, kv head) in chunks of kOutChunk:
+// first the chunk's probability-spectrum weights  w_k * Pf[g, k]  are formed from Zf (the unpacking
+// formula; one thread per bin) into shared memory, then the warps stream the coefficient rows, four
+// bins per warp in flight.  The last CTA of a (sequence, kv head) to finish sums the slice partials in
+// a fixed order, divides by P * colsum and writes the output rows.
 // grid = (slices, batch * H); block = 256.
+constexpr int kOutChunk = 256;
+
 template <typename TQ, int GQ, bool APPEND>
 __global__ void __launch_bounds__(kAttnWarps * 32)
-k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, const int32_t *__restrict__ t_len,
-               const float2 *__restrict__ Zf, const int32_t *__restrict__ bins, float *__restrict__ partial,
-               int M, int H, int HQ, fft::Geometry g, int bins_per_slice) {
+k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t *__restrict__ t_len,
+               const float2 *__restrict__ Zf, const float *__restrict__ colsum, const int32_t *__restrict__ bins,
+               float *__restrict__ partial, unsigned int *__restrict__ tickets, TQ *__restrict__ out,
+               int M, int H, int HQ, fft::Geometry g, int bins_per_slice, float inv_P) {
     using namespace fft;
-    __shared__ __align__(16) float red[kAttnWarps][GQ][kHeadDim];
+    // the weights of a chunk and the final cross-warp reduction share one buffer
+    constexpr size_t kWgtBytes = (size_t)kOutChunk * GQ * sizeof(float2) + (APPEND ? kOutChunk * sizeof(float2) : 0);
+    constexpr size_t kRedBytes = (size_t)kAttnWarps * GQ * kHeadDim * sizeof(float);
+    __shared__ __align__(16) unsigned char sbuf[kWgtBytes > kRedBytes ? kWgtBytes : kRedBytes];
+    float2 (*wgt)[GQ] = reinterpret_cast<float2 (*)[GQ]>(sbuf);                         // (w Re Pf, -w Im Pf) / bin
+    float2 *upd = reinterpret_cast<float2 *>(sbuf + (size_t)kOutChunk * GQ * sizeof(float2));   // APPEND: (cos, sin) of w k t
+    float (*red)[GQ][kHeadDim] = reinterpret_cast<float (*)[GQ][kHeadDim]>(sbuf);
+    __shared__ unsigned int last_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
     const int kbeg = blockIdx.x * bins_per_slice;
@@ -275,38 +346,68 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, const in
     float4 acc[GQ];
 #pragma unroll
     for (int q = 0; q < GQ; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k = kbeg + warp; k < kend; k += kAttnWarps) {
-        float *rp = base + (size_t)k * kHeadDim + lane * 4;
-        float4 re = ld_stream(rp);
-        float4 im = ld_stream(rp + plane);
-        const uint32_t bin = (uint32_t)bins[k];
-        if (APPEND) {
-            float c, s;
-            twiddle(phase_mod(bin, t, g.P), g.P, c, s);
-            re.x = fmaf(x.x, c, re.x); im.x = fmaf(-x.x, s, im.x);
-            re.y = fmaf(x.y, c, re.y); im.y = fmaf(-x.y, s, im.y);
-            re.z = fmaf(x.z, c, re.z); im.z = fmaf(-x.z, s, im.z);
-            re.w = fmaf(x.w, c, re.w); im.w = fmaf(-x.w, s, im.w);
-            st_stream(rp, re);
-            st_stream(rp + plane, im);
-        }
-        const float w = hermitian_weight(bin, g.P);
-        const int ka = (int)bin & (g.N - 1), kb = (g.N - ka) & (g.N - 1);
-        const float2 ph = unit_phasor(bin, g.P);
+
+    for (int c0 = kbeg; c0 < kend; c0 += kOutChunk) {
+        const int cn = min(kOutChunk, kend - c0);
+        __syncthreads();                             // previous chunk's weights are no longer read
+        if ((int)threadIdx.x < cn) {
+            const uint32_t bin = (uint32_t)bins[c0 + threadIdx.x];
+            const float w = 0.5f * hermitian_weight(bin, g.P);
+            const int ka = (int)bin & (g.N - 1), kb = (g.N - ka) & (g.N - 1);
+            const float2 ph = unit_phasor(bin, g.P);
+            const float2 *za_p = Zf + (size_t)ka * g.Gp + gcol, *zb_p = Zf + (size_t)kb * g.Gp + gcol;
 #pragma unroll
-        for (int q = 0; q < GQ; ++q) {
-            const float2 za = Zf[(size_t)ka * g.Gp + gcol + q];
-            float2 zb = Zf[(size_t)kb * g.Gp + gcol + q];
-            zb.y = -zb.y;
-            const float2 A = cadd(za, zb), D = csub(za, zb);             // 2A, 2jB
-            const float2 W = cadd(A, cmul(ph, make_float2(D.y, -D.x)));   // 2 Pf
-            const float ar = 0.5f * w * W.x, ai = -0.5f * w * W.y;
-            acc[q].x = fmaf(re.x, ar, fmaf(im.x, ai, acc[q].x));
-            acc[q].y = fmaf(re.y, ar, fmaf(im.y, ai, acc[q].y));
-            acc[q].z = fmaf(re.z, ar, fmaf(im.z, ai, acc[q].z));
-            acc[q].w = fmaf(re.w, ar, fmaf(im.w, ai, acc[q].w));
+            for (int q = 0; q < GQ; ++q) {
+                const float2 za = za_p[q];
+                float2 zb = zb_p[q];
+                zb.y = -zb.y;
+                const float2 A = cadd(za, zb), D = csub(za, zb);                 // 2A, 2jB
+                const float2 W = cadd(A, cmul(ph, make_float2(D.y, -D.x)));       // 2 Pf
+                wgt[threadIdx.x][q] = make_float2(w * W.x, -w * W.y);
+            }
+            if (APPEND) {
+                float cs, sn;
+                twiddle(phase_mod(bin, t, g.P), g.P, cs, sn);
+                upd[threadIdx.x] = make_float2(cs, sn);
+            }
+        }
+        __syncthreads();
+        for (int i0 = warp * 4; i0 < cn; i0 += kAttnWarps * 4) {
+            float4 re[4], im[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                re[u] = im[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (i0 + u < cn) {
+                    const float *rp = base + (size_t)(c0 + i0 + u) * kHeadDim + lane * 4;
+                    re[u] = ld_stream(rp);
+                    im[u] = ld_stream(rp + plane);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (i0 + u >= cn) continue;
+                if (APPEND) {
+                    const float2 cs = upd[i0 + u];
+                    re[u].x = fmaf(x.x, cs.x, re[u].x); im[u].x = fmaf(-x.x, cs.y, im[u].x);
+                    re[u].y = fmaf(x.y, cs.x, re[u].y); im[u].y = fmaf(-x.y, cs.y, im[u].y);
+                    re[u].z = fmaf(x.z, cs.x, re[u].z); im[u].z = fmaf(-x.z, cs.y, im[u].z);
+                    re[u].w = fmaf(x.w, cs.x, re[u].w); im[u].w = fmaf(-x.w, cs.y, im[u].w);
+                    float *wp = base + (size_t)(c0 + i0 + u) * kHeadDim + lane * 4;
+                    st_stream(wp, re[u]);
+                    st_stream(wp + plane, im[u]);
+                }
+#pragma unroll
+                for (int q = 0; q < GQ; ++q) {
+                    const float2 a = wgt[i0 + u][q];
+                    acc[q].x = fmaf(re[u].x, a.x, fmaf(im[u].x, a.y, acc[q].x));
+                    acc[q].y = fmaf(re[u].y, a.x, fmaf(im[u].y, a.y, acc[q].y));
+                    acc[q].z = fmaf(re[u].z, a.x, fmaf(im[u].z, a.y, acc[q].z));
+                    acc[q].w = fmaf(re[u].w, a.x, fmaf(im[u].w, a.y, acc[q].w));
+                }
+            }
         }
     }
+    __syncthreads();                                 // the last chunk's weights are no longer read
 #pragma unroll
     for (int q = 0; q < GQ; ++q) *reinterpret_cast<float4 *>(&red[warp][q][lane * 4]) = acc[q];
     __syncthreads();
@@ -317,46 +418,36 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, const in
         for (int w = 0; w < kAttnWarps; ++w) s += red[w][q][c];
         partial[(((size_t)bh * gridDim.x + blockIdx.x) * GQ + q) * kHeadDim + c] = s;
     }
-}
-
-// Sum the slice partials; softmax normaliser = sum_tiles sloc * exp(mloc - max mloc); convert.
-// With bump_batch > 0 the first block also advances the token counters (fused append).
-// grid = batch * H * GQ; block = 128.
-template <typename TOut>
-__global__ void __launch_bounds__(kHeadDim)
-k_attn_out_reduce_fft(const float *__restrict__ partial, const float *__restrict__ mloc, const float *__restrict__ sloc,
-                      int n_tiles, int Gp, TOut *__restrict__ out, int slices, int GQ, float inv_P,
-                      int32_t *__restrict__ t_len, int bump_batch) {
-    __shared__ float red[kHeadDim];
-    const int bh = blockIdx.x / GQ, q = blockIdx.x % GQ, c = threadIdx.x;
-    const int col = bh * GQ + q;                 // = sequence * HQ + head
-    float mx = -INFINITY;
-    for (int ti = c; ti < n_tiles; ti += kHeadDim) mx = fmaxf(mx, mloc[(size_t)ti * Gp + col]);
-    red[c] = mx;
+    // last CTA of this (sequence, kv head): reduce the slices in a fixed order
+    __threadfence();
     __syncthreads();
-    for (int s = kHeadDim / 2; s > 0; s >>= 1) {
-        if (c < s) red[c] = fmaxf(red[c], red[c + s]);
-        __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int prev = atomicAdd(&tickets[bh], 1u);
+        last_flag = prev == gridDim.x - 1 ? 1u : 0u;
+        if (last_flag) tickets[bh] = 0u;             // ready for the next call on this stream
     }
-    mx = red[0];
     __syncthreads();
-    float sum = 0.f;
-    for (int ti = c; ti < n_tiles; ti += kHeadDim) {
-        const float ml = mloc[(size_t)ti * Gp + col];
-        if (ml != -INFINITY) sum += sloc[(size_t)ti * Gp + col] * __expf(ml - mx);
+    if (last_flag) {
+        __threadfence();
+        for (int e = threadIdx.x; e < GQ * kHeadDim; e += blockDim.x) {
+            const int q = e / kHeadDim, c = e % kHeadDim;
+            float s = 0.f;
+            for (int sl = 0; sl < (int)gridDim.x; ++sl)
+                s += __ldcg(partial + (((size_t)bh * gridDim.x + sl) * GQ + q) * kHeadDim + c);
+            store1(out + (size_t)(gcol + q) * kHeadDim + c, s * inv_P / colsum[gcol + q]);
+        }
+        if (APPEND) {
+            // every CTA of this sequence has read t_len before taking its ticket; the last CTA of the
+            // sequence's last kv head advances the counter once all H heads are through
+            if (threadIdx.x == 0) {
+                const unsigned int done = atomicAdd(&tickets[gridDim.y + b], 1u);
+                if (done == (unsigned int)H - 1u) {
+                    tickets[gridDim.y + b] = 0u;
+                    t_len[b] += 1;
+                }
+            }
+        }
     }
-    red[c] = sum;
-    __syncthreads();
-    for (int s = kHeadDim / 2; s > 0; s >>= 1) {
-        if (c < s) red[c] += red[c + s];
-        __syncthreads();
-    }
-    const float colsum = red[0];
-    float s = 0.f;
-    for (int sl = 0; sl < slices; ++sl) s += partial[(((size_t)bh * slices + sl) * GQ + q) * kHeadDim + c];
-    store1(out + (size_t)col * kHeadDim + c, s * inv_P / colsum);
-    if (blockIdx.x == 0)
-        for (int i = c; i < bump_batch; i += kHeadDim) t_len[i] += 1;
 }
 
 }  // namespace faedkv

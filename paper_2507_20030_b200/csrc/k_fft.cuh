@@ -3,7 +3,7 @@
 //
 // A real length-P signal is handled as a complex signal of length N = P/2 (even samples in the real
 // part, odd samples in the imaginary part), and the complex length-N transform with kernel e^{+j2pi km/N}
-// is split as N = N1 * N2 into two passes of small shared-memory FFTs with one twiddle in between:
+// is split as N = N1 * N2 into two passes of small FFTs with one twiddle in between:
 //
 //   input index  k = N2*k1 + k2,   output index  m = m1 + N1*m2
 //   pass A (per k2, over k1):   Y[m1][k2] = e^{+j2pi k2 m1/N} * sum_k1 Z[N2 k1 + k2] e^{+j2pi k1 m1/N1}
@@ -14,9 +14,11 @@
 // Packed signal -> half spectrum of W[k] = sum_n p[n] e^{+j2pi kn/P}, with Zf = transform of p[2m] + j p[2m+1]:
 //   W[k] = (Zf[k'] + conj Zf[-k'])/2 + e^{+j2pi k/P} (Zf[k'] - conj Zf[-k'])/(2j),   k' = k mod N
 //
-// The in-shared-memory FFT is a mixed-radix (8, 4, 2) Stockham autosort over the rows of a
-// [rows][columns] tile, ping-ponging between two buffers; "columns" are independent signals
-// (query heads or channels) times however many transforms of the pass the CTA takes.
+// One small FFT (length NF = 2^LG <= 512, many independent columns side by side) is a Stockham
+// autosort of one to three register-resident butterflies of radix 4, 8 or 16: the first stage reads
+// its inputs straight from wherever they are (global memory, a gather, another shared-memory tile),
+// the last stage hands its outputs to a store functor, and only the exchange between stages goes
+// through shared memory.
 #pragma once
 #include "common.cuh"
 
@@ -25,7 +27,8 @@ namespace fft {
 
 constexpr int kThreads = 256;
 constexpr int kCW = 16;            // independent signals (columns) per CTA
-constexpr int kTileMax = 4096;     // complex elements of one shared-memory tile (32 KB; two tiles ping-pong)
+constexpr int kLgCW = 4;
+constexpr int kTileMax = 4096;     // complex elements of one shared-memory tile (32 KB) when NF * 16 allows
 
 __host__ __device__ constexpr int ilog2(int v) { return v <= 1 ? 0 : 1 + ilog2(v >> 1); }
 
@@ -49,7 +52,7 @@ inline Geometry make_geometry(int P, int G) {
     g.Gp = (G + kCW - 1) / kCW * kCW;
     return g;
 }
-// P is a power of two whose two passes fit the shared-memory tiles.
+// P is a power of two whose two passes fit the shared-memory tiles (3 <= lgN1 <= 9, 2 <= lgN2 <= 9).
 inline bool supported(int P) { return P >= 64 && P <= (1 << 19) && (P & (P - 1)) == 0; }
 
 // How many transforms of a pass one CTA takes (a power of two): fill the tile, but keep at least
@@ -60,7 +63,6 @@ inline int transforms_per_cta(int rows, int n_transforms, int col_blocks) {
     while (kt > 1 && (kt > n_transforms || (n_transforms / kt) * col_blocks < 2 * 148)) kt >>= 1;
     return kt;
 }
-inline size_t smem_bytes(int rows, int kt) { return (size_t)(2 * rows * kt * kCW + rows) * sizeof(float2); }
 
 __device__ __forceinline__ float2 cmul(float2 a, float2 b) {
     return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
@@ -81,7 +83,8 @@ __device__ __forceinline__ void fill_twiddles(float2 *tw, int NF) {
     for (int i = threadIdx.x; i < NF; i += kThreads) tw[i] = unit_phasor((uint32_t)i, (uint32_t)NF);
 }
 
-// Natural-order DFTs of size 2, 4, 8 with kernel e^{+j 2 pi kr / R}.
+// ---- register butterflies: DFT of size R with kernel e^{+j 2 pi kr / R} ----------------------------------
+// Output r of the DFT is left in v[perm<R>(r)] (identity except for R = 16).
 __device__ __forceinline__ void dft2(float2 &a, float2 &b) {
     const float2 t = a;
     a = cadd(t, b);
@@ -111,54 +114,87 @@ template <> __device__ __forceinline__ void dft<8>(float2 (&v)[8]) {
     v[2] = cadd(e2, o2); v[6] = csub(e2, o2);
     v[3] = cadd(e3, o3); v[7] = csub(e3, o3);
 }
+// 16 = 4 x 4: n = n1 + 4 n2, k = k2 + 4 k1; X[k2 + 4 k1] ends in v[k1 + 4 k2].
+template <> __device__ __forceinline__ void dft<16>(float2 (&v)[16]) {
+#pragma unroll
+    for (int n1 = 0; n1 < 4; ++n1) dft4(v[n1], v[n1 + 4], v[n1 + 8], v[n1 + 12]);   // v[n1 + 4 k2] = A[n1][k2]
+    const float c1 = 0.92387953251128674f, s1 = 0.38268343236508977f, h = 0.70710678118654752f;
+    // v[n1 + 4 k2] *= e^{+j 2 pi n1 k2 / 16}
+    v[5] = cmul(v[5], make_float2(c1, s1));                                   // n1 k2 = 1
+    v[6] = make_float2(h * (v[6].x - v[6].y), h * (v[6].x + v[6].y));         // 2
+    v[7] = cmul(v[7], make_float2(s1, c1));                                   // 3
+    v[9] = make_float2(h * (v[9].x - v[9].y), h * (v[9].x + v[9].y));         // 2
+    v[10] = cmulj(v[10]);                                                     // 4
+    v[11] = make_float2(-h * (v[11].x + v[11].y), h * (v[11].x - v[11].y));   // 6
+    v[13] = cmul(v[13], make_float2(s1, c1));                                 // 3
+    v[14] = make_float2(-h * (v[14].x + v[14].y), h * (v[14].x - v[14].y));   // 6
+    v[15] = cmul(v[15], make_float2(-c1, -s1));                               // 9
+#pragma unroll
+    for (int k2 = 0; k2 < 4; ++k2) dft4(v[4 * k2], v[4 * k2 + 1], v[4 * k2 + 2], v[4 * k2 + 3]);
+}
+template <int R> __device__ __forceinline__ constexpr int perm(int r) { return R == 16 ? ((r >> 2) | ((r & 3) << 2)) : r; }
 
-// One Stockham stage of radix R over a [NF][cols] tile; Ns = product of the radices already applied.
-template <int R>
-__device__ __forceinline__ void fft_stage(const float2 *__restrict__ in, float2 *__restrict__ out,
-                                          const float2 *__restrict__ tw, int NF, int Ns, int lg_cols) {
-    const int stride = (NF / R) << lg_cols;      // elements between the R inputs of a butterfly
-    const int tw_step = NF / (Ns * R);
-    for (int it = threadIdx.x; it < stride; it += kThreads) {
+// Radices of the stages of a length-2^LG transform.
+template <int LG> struct Radix;
+template <> struct Radix<2> { static constexpr int R1 = 4, R2 = 1, R3 = 1; };
+template <> struct Radix<3> { static constexpr int R1 = 8, R2 = 1, R3 = 1; };
+template <> struct Radix<4> { static constexpr int R1 = 16, R2 = 1, R3 = 1; };
+template <> struct Radix<5> { static constexpr int R1 = 4, R2 = 8, R3 = 1; };
+template <> struct Radix<6> { static constexpr int R1 = 8, R2 = 8, R3 = 1; };
+template <> struct Radix<7> { static constexpr int R1 = 8, R2 = 16, R3 = 1; };
+template <> struct Radix<8> { static constexpr int R1 = 16, R2 = 16, R3 = 1; };
+template <> struct Radix<9> { static constexpr int R1 = 8, R2 = 8, R3 = 8; };
+// Shared-memory exchange buffers a transform of length 2^lg needs (each rows * columns float2).
+__host__ __device__ constexpr int exchange_buffers(int lg) { return lg >= 9 ? 2 : (lg >= 5 ? 1 : 0); }
+
+// One Stockham stage of radix R over NF rows x (1 << lg_cols) columns; NS = product of the radices
+// already applied.  in(row, col) -> float2, out(row, col, value).
+template <int NF, int R, int NS, typename In, typename Out>
+__device__ __forceinline__ void fft_stage(int lg_cols, const float2 *__restrict__ tw, In in, Out out) {
+    constexpr int NB = NF / R;          // butterflies per column; also the row stride of a butterfly's inputs
+    const int items = NB << lg_cols;
+    for (int it = threadIdx.x; it < items; it += kThreads) {
         const int c = it & ((1 << lg_cols) - 1), j = it >> lg_cols;
-        const int k = j & (Ns - 1);
         float2 v[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) v[r] = in[it + r * stride];
-        if (Ns > 1) {
+        for (int r = 0; r < R; ++r) v[r] = in(j + r * NB, c);
+        const int k = j & (NS - 1);
+        if (NS > 1) {
 #pragma unroll
-            for (int r = 1; r < R; ++r) v[r] = cmul(v[r], tw[k * r * tw_step]);
+            for (int r = 1; r < R; ++r) v[r] = cmul(v[r], tw[k * r * (NF / (NS * R))]);
         }
         dft<R>(v);
         const int j0 = (j - k) * R + k;
 #pragma unroll
-        for (int r = 0; r < R; ++r) out[((j0 + r * Ns) << lg_cols) + c] = v[r];
+        for (int r = 0; r < R; ++r) out(j0 + perm<R>(r) * NS, c, v[r]);
     }
 }
 
-// FFT over the rows of the tile in `a` (scratch `b`, same size); returns the buffer holding the result.
-// Every thread of the CTA must call it; it ends with a __syncthreads().
-__device__ __forceinline__ float2 *fft_tile(float2 *a, float2 *b, const float2 *tw, int NF, int lg_cols) {
-    const int lg = 31 - __clz(NF);
-    int Ns = 1;
-    const int rem = lg % 3;
-    if (rem == 1) {
-        fft_stage<2>(a, b, tw, NF, Ns, lg_cols);
-        Ns = 2;
-    } else if (rem == 2) {
-        fft_stage<4>(a, b, tw, NF, Ns, lg_cols);
-        Ns = 4;
-    }
-    if (rem != 0) {
+// Length-2^LG transform over the rows of a tile of (1 << lg_cols) columns.  load(row, col) supplies the
+// inputs, store(row, col, value) takes the outputs; xa, xb are the exchange buffers (see
+// exchange_buffers()), tw the NF-entry twiddle table.  All threads of the CTA must call it; it
+// contains __syncthreads() between stages but none before the first or after the last stage.
+template <int LG, typename Load, typename Store>
+__device__ __forceinline__ void fft_rows(int lg_cols, float2 *xa, float2 *xb, const float2 *tw, Load load, Store store) {
+    constexpr int NF = 1 << LG;
+    constexpr int R1 = Radix<LG>::R1, R2 = Radix<LG>::R2, R3 = Radix<LG>::R3;
+    auto rd_a = [&](int row, int c) { return xa[(row << lg_cols) + c]; };
+    auto wr_a = [&](int row, int c, float2 v) { xa[(row << lg_cols) + c] = v; };
+    auto rd_b = [&](int row, int c) { return xb[(row << lg_cols) + c]; };
+    auto wr_b = [&](int row, int c, float2 v) { xb[(row << lg_cols) + c] = v; };
+    if constexpr (R2 == 1) {
+        fft_stage<NF, R1, 1>(lg_cols, tw, load, store);
+    } else if constexpr (R3 == 1) {
+        fft_stage<NF, R1, 1>(lg_cols, tw, load, wr_a);
         __syncthreads();
-        float2 *t = a; a = b; b = t;
-    }
-    while (Ns < NF) {
-        fft_stage<8>(a, b, tw, NF, Ns, lg_cols);
-        Ns *= 8;
+        fft_stage<NF, R2, R1>(lg_cols, tw, rd_a, store);
+    } else {
+        fft_stage<NF, R1, 1>(lg_cols, tw, load, wr_a);
         __syncthreads();
-        float2 *t = a; a = b; b = t;
+        fft_stage<NF, R2, R1>(lg_cols, tw, rd_a, wr_b);
+        __syncthreads();
+        fft_stage<NF, R3, R1 * R2>(lg_cols, tw, rd_b, store);
     }
-    return a;
 }
 
 // Element (m1, row, col) of the intermediate array between the two passes: [N1][N2][Gp] float2.
