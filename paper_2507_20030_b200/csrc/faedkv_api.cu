@@ -632,8 +632,9 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     ctx->gq = gq;
     ctx->hqp = (cfg->n_q_heads + 31) / 32 * 32;
     ctx->use_tc = cfg->kv_dtype == FAEDKV_BF16 && cfg->decode_mode != FAEDKV_DECODE_SIMT;
-    ctx->use_fft = fft::supported(cfg->n_dft) &&
-                   (cfg->decode_mode == FAEDKV_DECODE_AUTO || cfg->decode_mode == FAEDKV_DECODE_FFT);
+    const bool fft_ok = fft::supported(cfg->n_dft) && fft::fits_32bit_index(cfg->n_dft, cfg->max_batch * cfg->n_q_heads);
+    if (cfg->decode_mode == FAEDKV_DECODE_FFT && !fft_ok) { delete ctx; return FAEDKV_ERR_UNSUPPORTED; }
+    ctx->use_fft = fft_ok && (cfg->decode_mode == FAEDKV_DECODE_AUTO || cfg->decode_mode == FAEDKV_DECODE_FFT);
     ctx->plans.resize(cfg->n_layers);
     if (cudaGetDevice(&ctx->device) != cudaSuccess ||
         cudaMalloc(&ctx->tick, sizeof(unsigned int) * (cfg->n_layers + 1)) != cudaSuccess ||

@@ -116,8 +116,8 @@ k_afft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float2 *__
         float2 z = make_float2(0.f, 0.f);
         const int sa = slot[k], sb = slot[g.N - k];
         if ((sa >= 0 || sb >= 0) && col < g.G) {
-            const float2 xk = sa >= 0 ? Qs[(size_t)sa * g.Gp + col] : make_float2(0.f, 0.f);
-            float2 xm = sb >= 0 ? Qs[(size_t)sb * g.Gp + col] : make_float2(0.f, 0.f);
+            const float2 xk = sa >= 0 ? Qs[(uint32_t)sa * (uint32_t)g.Gp + (uint32_t)col] : make_float2(0.f, 0.f);
+            float2 xm = sb >= 0 ? Qs[(uint32_t)sb * (uint32_t)g.Gp + (uint32_t)col] : make_float2(0.f, 0.f);
             xm.y = -xm.y;                                            // conj X[N-k]
             z = cadd(cadd(xk, xm), cmulj(cmul(tab_p[(k1 << lgKT) + kt], csub(xk, xm))));
         }
@@ -287,7 +287,7 @@ k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restr
         return make_float2(v.x * f, v.y * f);
     };
     auto store = [&](int k2p, int cidx, float2 v) {
-        Zf[((size_t)(k1_0 + (cidx >> kLgCW)) + (size_t)g.N2 * k2p) * g.Gp + g0 + (cidx & (kCW - 1))] = v;
+        Zf[((uint32_t)(k1_0 + (cidx >> kLgCW)) + (uint32_t)g.N2 * (uint32_t)k2p) * (uint32_t)g.Gp + (uint32_t)(g0 + (cidx & (kCW - 1)))] = v;
     };
     fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
 }
@@ -355,7 +355,7 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
             const float w = 0.5f * hermitian_weight(bin, g.P);
             const int ka = (int)bin & (g.N - 1), kb = (g.N - ka) & (g.N - 1);
             const float2 ph = unit_phasor(bin, g.P);
-            const float2 *za_p = Zf + (size_t)ka * g.Gp + gcol, *zb_p = Zf + (size_t)kb * g.Gp + gcol;
+            const float2 *za_p = Zf + (uint32_t)ka * (uint32_t)g.Gp + gcol, *zb_p = Zf + (uint32_t)kb * (uint32_t)g.Gp + gcol;
 #pragma unroll
             for (int q = 0; q < GQ; ++q) {
                 const float2 za = za_p[q];

@@ -198,8 +198,14 @@ __device__ __forceinline__ void fft_rows(int lg_cols, float2 *xa, float2 *xb, co
 }
 
 // Element (m1, row, col) of the intermediate array between the two passes: [N1][N2][Gp] float2.
-__device__ __forceinline__ size_t y_index(const Geometry &g, int m1, int row, int col) {
-    return ((size_t)m1 * g.N2 + row) * g.Gp + col;
+// 32-bit on purpose (address arithmetic is a visible share of these kernels' instructions): the host
+// only takes the FFT-shaped path while N * Gp < 2^31.
+__device__ __forceinline__ uint32_t y_index(const Geometry &g, int m1, int row, int col) {
+    return ((uint32_t)m1 * (uint32_t)g.N2 + (uint32_t)row) * (uint32_t)g.Gp + (uint32_t)col;
+}
+inline bool fits_32bit_index(int P, int G) {
+    const Geometry g = make_geometry(P, G);
+    return (unsigned long long)g.N * (unsigned long long)g.Gp < (1ull << 31);
 }
 
 }  // namespace fft
