@@ -168,6 +168,87 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+
+# --------------------------------------------------------------------------------------- decode sections
+DECODE_WORKLOADS = [
+    dict(name="configs[2]: streaming decode, batch 16, prefill 16384 tokens at 1/8 retention", config=2,
+         n_layers=32, n_kv_heads=8, n_q_heads=32, batch=16, T=16384, M=2048),
+    dict(name="configs[3]: long context, batch 1, 131072 tokens at 1/16 retention", config=3,
+         n_layers=32, n_kv_heads=8, n_q_heads=32, batch=1, T=131072, M=8192),
+]
+
+
+def decode_section(torch, binding, synth, dev, W, peaks, iters):
+    """Decode us / layer / step at one workload shape: the state comes from a real prefill (one layer of
+    K/V resident at a time), then the three decode calls are timed over all layers, each loop replayed
+    as one CUDA graph (launch gaps excluded) and, for the fused call, also launched eagerly."""
+    NL, H, HQ, B, T, M = (W[k] for k in ("n_layers", "n_kv_heads", "n_q_heads", "batch", "T", "M"))
+    P, D = T, 128
+    ctx = binding.Context(n_layers=NL, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=binding.BF16)
+    seed = synth.config_seed(W["config"])
+    cKs, cVs, tls = [], [], []
+    for l in range(NL):
+        ctx.plan(l, binding.mask_mixed(P, M, l, seed))
+        K, V = synth.make_kv(synth.config_seed(W["config"], l), B, H, T, D, dtype=torch.bfloat16, device=dev)
+        cK, cV = ctx.alloc_coef(l, B, device=dev), ctx.alloc_coef(l, B, device=dev)
+        tl = torch.zeros(B, dtype=torch.int32, device=dev)
+        ctx.compress_prefill(l, K, V, cK, cV, tl)
+        cKs.append(cK); cVs.append(cV); tls.append(tl)
+        torch.cuda.synchronize()
+        del K, V
+    k_new, v_new = synth.make_token(seed, 0, B, H, D, pos=T, dtype=torch.bfloat16, device=dev)
+    q = synth.make_q(seed, 0, B, HQ, D, dtype=torch.bfloat16, device=dev)
+    out = torch.empty((B, HQ, D), dtype=torch.bfloat16, device=dev)
+    loops = {
+        "append": lambda: [ctx.append(l, k_new, v_new, cKs[l], cVs[l], tls[l]) for l in range(NL)],
+        "decode_attn": lambda: [ctx.decode_attn(l, q, cKs[l], cVs[l], tls[l], out) for l in range(NL)],
+        "append_decode_attn": lambda: [ctx.append_decode_attn(l, k_new, v_new, q, cKs[l], cVs[l], tls[l], out)
+                                       for l in range(NL)],
+    }
+    coef_bytes = 2 * B * H * 2 * M * D * 4                      # K and V planes of one layer
+    alg_bytes = {"append": 2 * coef_bytes, "decode_attn": coef_bytes, "append_decode_attn": 2 * coef_bytes}
+    res = {"workload": W["name"], "iters": iters, "planes_bytes_per_layer": coef_bytes,
+           "l2": "32 layers cycled: %.0f MiB of planes per layer" % (coef_bytes / 2 ** 20)}
+    side = torch.cuda.Stream()
+    for name, fn in loops.items():
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        eager_us = a.elapsed_time(b) / iters / NL * 1e3
+        graph = torch.cuda.CUDAGraph()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.synchronize()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(iters):
+            graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) / iters / NL * 1e3
+        gbs = alg_bytes[name] / (us * 1e-6) / 1e9
+        res[name] = {"us": us, "us_eager_launches": eager_us, "bytes": alg_bytes[name], "bound": "hbm", "achieved": gbs,
+                     "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"]}
+    res["decode_us_per_layer_step"] = res["append_decode_attn"]["us"]
+    res["decode_us_per_layer_step_two_calls"] = res["append"]["us"] + res["decode_attn"]["us"]
+    if ctx.device_status() != 0:
+        raise RuntimeError("a kernel reported a device-side timeout; the numbers are invalid")
+    ctx.close()
+    del cKs, cVs
+    torch.cuda.empty_cache()
+    return res
+
 # --------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -334,6 +415,16 @@ def run_ours(args):
                "what": "phase A through the C ABI with pinned host K/V in and host coefficient planes out"}
         del hK, hV, hcK, hcV
 
+    # ---- decode at the workloads that define it (streaming decode, long context)
+    decode_sections = []
+    if not args.no_decode_configs and not args.layers:
+        del Ks, Vs, cKs, cVs, Ko, Vo
+        ctx.close()
+        torch.cuda.empty_cache()
+        for DW in DECODE_WORKLOADS:
+            decode_sections.append(decode_section(torch, binding, synth, dev, DW, peaks, args.decode_config_iters))
+    barrier()
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -351,7 +442,10 @@ def run_ours(args):
         # float32 FMA pipe: 148 SMs x 128 lanes x 2 FLOP x 1.965 GHz
         peak_tf, bound = 148 * 128 * 2 * 1.965e9 / 1e12, "alu"
     roofline = {"kernel": "prefill transform (" + mode + ")", "bound": bound, "achieved": achieved_tf,
-                "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf, "traffic": None,
+                "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
+                # ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel at this size
+                # (profiles/k_prefill_umma_T32768_M4096.md); the kernel is unchanged since that capture
+                "traffic": 191.4e6 if (mode == "tcgen05-bf16" and (args.twiddle_terms or 1) == 1) else None,
                 "peak_source": peaks["source"] + (" bf16 sustained" if bound == "tensor" else " (derived f32 FMA peak)"),
                 "flop_per_launch": flop_per_launch, "launch_ms": prefill_launch_ms,
                 "mma_passes": (args.twiddle_terms if args.twiddle_terms else 1) if bound == "tensor" else None}
@@ -379,6 +473,12 @@ def run_ours(args):
         "decode_iters": n_dec,
     }
 
+    decode["what"] = "configs[1] shape (batch 1), calls launched eagerly with events around each"
+    if decode_sections:
+        decode["configs"] = decode_sections
+        # the headline decode number is the streaming-decode workload's
+        decode["decode_us_per_layer_step_configs1_shape"] = decode["decode_us_per_layer_step"]
+        decode["decode_us_per_layer_step"] = decode_sections[0]["decode_us_per_layer_step"]
     line = {"metric": METRIC, "value": world * B * T / (prefill_ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -409,6 +509,9 @@ def main():
                     help="run only the first N layers of the workload (small case for profiler captures; "
                          "a bench value must use the default = all layers)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-decode-configs", action="store_true",
+                    help="skip the decode sections at the configs[2] and configs[3] shapes")
+    ap.add_argument("--decode-config-iters", type=int, default=10)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
