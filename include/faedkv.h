@@ -59,9 +59,13 @@ typedef enum {
 
 /* How the prefill transform is evaluated (faedkv_config.prefill_mode). */
 typedef enum {
-    FAEDKV_PREFILL_AUTO = 0,  /* bf16 K/V: tensor-core path; float32 K/V: float32 SIMT path */
+    FAEDKV_PREFILL_AUTO = 0,  /* bf16 K/V: tensor-core contraction; float32 K/V: FFT-shaped when P is a
+                                 power of two in [64, 2^19] (and decode_mode allows FFT), else float32 SIMT */
     FAEDKV_PREFILL_SIMT = 1,  /* float32 FMA contraction, twiddles exact to float32     */
-    FAEDKV_PREFILL_UMMA = 2   /* tcgen05 tensor-core contraction, bf16 operands, float32 accumulate */
+    FAEDKV_PREFILL_UMMA = 2,  /* tcgen05 tensor-core contraction, bf16 operands, float32 accumulate */
+    FAEDKV_PREFILL_FFT = 3    /* float32 two-pass FFT of every channel, then a gather of the retained
+                                 bins (power-of-two P; needs decode_mode AUTO or FFT): O(T log T) per
+                                 channel instead of O(T * M), float32-exact                          */
 } faedkv_prefill_mode;
 
 /* How reconstruction and the two transforms inside decode attention are evaluated

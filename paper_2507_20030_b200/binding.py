@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "lib", "libfaedkv.so")
 
 F32, BF16 = 0, 1
-PREFILL_AUTO, PREFILL_SIMT, PREFILL_UMMA = 0, 1, 2
+PREFILL_AUTO, PREFILL_SIMT, PREFILL_UMMA, PREFILL_FFT = 0, 1, 2, 3
 DECODE_AUTO, DECODE_SIMT, DECODE_UMMA, DECODE_FFT = 0, 1, 2, 3
 
 EXPORTS = [

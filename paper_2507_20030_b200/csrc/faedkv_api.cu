@@ -16,6 +16,8 @@
 #include "k_idft_umma.cuh"
 #include "k_attn_umma.cuh"
 #include "k_attn_fft.cuh"
+#include "k_recon_fft.cuh"
+#include "k_prefill_fft.cuh"
 
 using namespace faedkv;
 
@@ -41,10 +43,13 @@ struct TcScratch {
 // Scratch of the FFT-shaped decode attention (power-of-two P).
 struct FftScratch {
     float2 *Qs = nullptr, *Y = nullptr, *Zf = nullptr;
+    float2 *Yr = nullptr;                 // two-pass array of the FFT-shaped reconstruction / prefill, [N][recon_units * 128]
+    float2 *Zr = nullptr;                 // second array of the FFT-shaped prefill (full spectrum before the gather)
+    int recon_units = 0;                  // units (sequence, kv head) per launch group of the reconstruction
     float *mloc = nullptr, *sloc = nullptr, *colsum = nullptr;
     unsigned int *tickets = nullptr;      // [max_batch * H + max_batch], zero between calls
     int max_M = 0;
-    unsigned int attr_mask[3] = {0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
+    unsigned int attr_mask[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
 };
 
 }  // namespace
@@ -65,7 +70,8 @@ struct faedkv_ctx {
     UmmaPrefillState umma;             // tensor maps etc. of the tensor-core prefill
     TcScratch tc;
     bool use_tc = false;               // bf16 tensors and decode_mode != SIMT
-    bool use_fft = false;              // power-of-two P: FFT-shaped transforms in decode attention
+    bool use_fft = false;              // power-of-two P: FFT-shaped transforms in decode attention and reconstruction
+    bool prefill_fft = false;          // FFT-shaped prefill transform
     FftScratch fs;
     unsigned long long launches = 0;   // kernels enqueued by this context so far
     std::string err;
@@ -148,7 +154,7 @@ void free_scratch(faedkv_ctx *ctx) {
     cudaFree(t.cmax); cudaFree(t.psum); cudaFree(t.colsum); cudaFree(t.PfS);
     t = TcScratch();
     FftScratch &f = ctx->fs;
-    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.tickets);
+    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr);
     f = FftScratch();
 }
 
@@ -189,6 +195,16 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             const size_t n_tickets = (size_t)c.max_batch * c.n_kv_heads + c.max_batch;
             CUDA_TRY(ctx, cudaMalloc(&f.tickets, n_tickets * sizeof(unsigned int)));
             CUDA_TRY(ctx, cudaMemset(f.tickets, 0, n_tickets * sizeof(unsigned int)));
+            // reconstruction / FFT-shaped prefill: units per launch group, bounded by a 128 MB two-pass array.
+            // (These kernels are instruction-bound, not bandwidth-bound: measured, larger launches win over
+            // keeping the array L2-resident, up to about this size.)
+            const size_t unit_bytes = (size_t)g.N * kHeadDim * sizeof(float2);
+            size_t ru = (128u << 20) / unit_bytes;
+            if (ru < 1) ru = 1;
+            if (ru > (size_t)c.max_batch * c.n_kv_heads) ru = (size_t)c.max_batch * c.n_kv_heads;
+            f.recon_units = (int)ru;
+            CUDA_TRY(ctx, cudaMalloc(&f.Yr, ru * unit_bytes));
+            if (ctx->prefill_fft) CUDA_TRY(ctx, cudaMalloc(&f.Zr, ru * unit_bytes));
         }
         if (M > f.max_M) {
             cudaFree(f.Qs);
@@ -218,9 +234,11 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
                 CUDA_TRY(ctx, cudaMemset(t.Qf16, 0, 2 * (size_t)M * G * sizeof(__half)));   // padded columns stay finite
                 CUDA_TRY(ctx, cudaMalloc(&t.PfS, (size_t)kSplitsCap * 2 * M * G * sizeof(float)));
             }
-            const size_t cbytes = B * c.n_kv_heads * 2 * (size_t)M * kHeadDim * sizeof(__half);
-            CUDA_TRY(ctx, cudaMalloc(&t.C16K, cbytes));
-            CUDA_TRY(ctx, cudaMalloc(&t.C16V, cbytes));
+            if (!ctx->use_fft) {   // f16 copies of the planes: operands of the tensor-core reconstruction
+                const size_t cbytes = B * c.n_kv_heads * 2 * (size_t)M * kHeadDim * sizeof(__half);
+                CUDA_TRY(ctx, cudaMalloc(&t.C16K, cbytes));
+                CUDA_TRY(ctx, cudaMalloc(&t.C16V, cbytes));
+            }
             t.max_M = M;
         }
     }
@@ -400,6 +418,105 @@ int fft_opt_in(faedkv_ctx *ctx, K kernel, size_t bytes, unsigned int &done_mask,
     if (bytes <= 48 * 1024 || (done_mask >> lg) & 1u) return FAEDKV_OK;
     if (int r = opt_in_smem(ctx, kernel, (uint32_t)bytes)) return r;
     done_mask |= 1u << lg;
+    return FAEDKV_OK;
+}
+
+// FFT-shaped reconstruction of one tensor: pairs of (pass A, pass B) launches over runs of units.
+template <typename TOut>
+int launch_reconstruct_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const float *coef, const int32_t *t_len, int units,
+                                  int L, void *out, cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    FftScratch &f = ctx->fs;
+    constexpr int kOutKind = sizeof(TOut) == 2 ? 4 : 5;
+    for (int u0 = 0; u0 < units; u0 += f.recon_units) {
+        const int uc = units - u0 < f.recon_units ? units - u0 : f.recon_units;
+        const fft::Geometry g = fft::make_geometry(c.n_dft, uc * kHeadDim);
+        const int col_blocks = g.Gp / fft::kCW;
+        const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks));
+        const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks));
+        int rc = FAEDKV_ERR_UNSUPPORTED;
+        {
+            const dim3 grid(g.N2 >> lgKT, col_blocks);
+            const size_t smem = afft_smem_a(g.lgN1, lgKT, true);
+#define CALL(LG)                                                                                         \
+            rc = fft_opt_in(ctx, k_rfft_inv_a<LG>, smem, f.attr_mask[3], LG);                            \
+            if (rc == 0) k_rfft_inv_a<LG><<<grid, fft::kThreads, smem, st>>>(g, p.d_slot, coef, p.M, u0, f.Yr, lgKT)
+            FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
+#undef CALL
+            if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
+            if (int r = launch_check(ctx, "k_rfft_inv_a")) return r;
+        }
+        rc = FAEDKV_ERR_UNSUPPORTED;
+        {
+            const dim3 grid(g.N1 >> lgMT, col_blocks);
+            const size_t smem = rfft_smem_b(g.lgN2, lgMT);
+#define CALL(LG)                                                                                         \
+            rc = fft_opt_in(ctx, k_rfft_inv_b<LG, TOut>, smem, f.attr_mask[kOutKind], LG);               \
+            if (rc == 0) k_rfft_inv_b<LG, TOut><<<grid, fft::kThreads, smem, st>>>(g, f.Yr, t_len, c.n_kv_heads, u0, L, static_cast<TOut *>(out), lgMT)
+            FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
+#undef CALL
+            if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
+            if (int r = launch_check(ctx, "k_rfft_inv_b")) return r;
+        }
+    }
+    return FAEDKV_OK;
+}
+
+template <typename TOut>
+int launch_reconstruct_fft(faedkv_ctx *ctx, const LayerPlan &p, const float *coefK, const float *coefV, const int32_t *t_len,
+                           int batch, int L, void *K_out, void *V_out, cudaStream_t st) {
+    const int units = batch * ctx->cfg.n_kv_heads;
+    if (coefK != nullptr)
+        if (int r = launch_reconstruct_fft_tensor<TOut>(ctx, p, coefK, t_len, units, L, K_out, st)) return r;
+    if (coefV != nullptr)
+        if (int r = launch_reconstruct_fft_tensor<TOut>(ctx, p, coefV, t_len, units, L, V_out, st)) return r;
+    return FAEDKV_OK;
+}
+
+// FFT-shaped prefill of one tensor: (pass A', pass B', gather) over runs of units.
+template <typename TIn>
+int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x, int units, int T, float *coef,
+                              cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    FftScratch &f = ctx->fs;
+    constexpr int kInKind = sizeof(TIn) == 2 ? 6 : 7;
+    const int per = f.recon_units > 1 ? f.recon_units / 2 : 1;      // two arrays live at once: half the units each
+    for (int u0 = 0; u0 < units; u0 += per) {
+        const int uc = units - u0 < per ? units - u0 : per;
+        const fft::Geometry g = fft::make_geometry(c.n_dft, uc * kHeadDim);
+        const int col_blocks = g.Gp / fft::kCW;
+        const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks));
+        const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks));
+        int rc = FAEDKV_ERR_UNSUPPORTED;
+        {
+            const dim3 grid(g.N1 >> lgMT, col_blocks);
+            const size_t smem = pfft_smem_a(g.lgN2, lgMT);
+#define CALL(LG)                                                                                         \
+            rc = fft_opt_in(ctx, k_pfft_fwd_a<LG, TIn>, smem, f.attr_mask[kInKind], LG);                 \
+            if (rc == 0) k_pfft_fwd_a<LG, TIn><<<grid, fft::kThreads, smem, st>>>(g, static_cast<const TIn *>(x), T, u0, f.Yr, lgMT)
+            FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
+#undef CALL
+            if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
+            if (int r = launch_check(ctx, "k_pfft_fwd_a")) return r;
+        }
+        rc = FAEDKV_ERR_UNSUPPORTED;
+        {
+            const dim3 grid(g.N2 >> lgKT, col_blocks);
+            const size_t smem = pfft_smem_b(g.lgN1, lgKT);
+#define CALL(LG)                                                                                         \
+            rc = fft_opt_in(ctx, k_pfft_fwd_b<LG>, smem, f.attr_mask[8], LG);                            \
+            if (rc == 0) k_pfft_fwd_b<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Yr, f.Zr, lgKT)
+            FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
+#undef CALL
+            if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
+            if (int r = launch_check(ctx, "k_pfft_fwd_b")) return r;
+        }
+        {
+            const dim3 grid((p.M + 7) / 8, uc);
+            k_pfft_gather<<<grid, 256, 0, st>>>(g, f.Zr, p.d_bins, p.M, u0, coef);
+            if (int r = launch_check(ctx, "k_pfft_gather")) return r;
+        }
+    }
     return FAEDKV_OK;
 }
 
@@ -615,7 +732,7 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
         cfg->n_dft < 2 || cfg->n_dft > (1 << 24))
         return FAEDKV_ERR_INVALID_ARG;
     if (cfg->kv_dtype != FAEDKV_F32 && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_INVALID_ARG;
-    if (cfg->prefill_mode < FAEDKV_PREFILL_AUTO || cfg->prefill_mode > FAEDKV_PREFILL_UMMA) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->prefill_mode < FAEDKV_PREFILL_AUTO || cfg->prefill_mode > FAEDKV_PREFILL_FFT) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->twiddle_terms < 0 || cfg->twiddle_terms > 2) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->decode_mode < FAEDKV_DECODE_AUTO || cfg->decode_mode > FAEDKV_DECODE_FFT) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->decode_mode == FAEDKV_DECODE_UMMA && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_UNSUPPORTED;
@@ -635,6 +752,10 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     const bool fft_ok = fft::supported(cfg->n_dft) && fft::fits_32bit_index(cfg->n_dft, cfg->max_batch * cfg->n_q_heads);
     if (cfg->decode_mode == FAEDKV_DECODE_FFT && !fft_ok) { delete ctx; return FAEDKV_ERR_UNSUPPORTED; }
     ctx->use_fft = fft_ok && (cfg->decode_mode == FAEDKV_DECODE_AUTO || cfg->decode_mode == FAEDKV_DECODE_FFT);
+    // the FFT-shaped prefill shares the decode path's scratch, so it needs that path too
+    if (cfg->prefill_mode == FAEDKV_PREFILL_FFT && !ctx->use_fft) { delete ctx; return FAEDKV_ERR_UNSUPPORTED; }
+    ctx->prefill_fft = ctx->use_fft && (cfg->prefill_mode == FAEDKV_PREFILL_FFT ||
+                                        (cfg->prefill_mode == FAEDKV_PREFILL_AUTO && cfg->kv_dtype == FAEDKV_F32));
     ctx->plans.resize(cfg->n_layers);
     if (cudaGetDevice(&ctx->device) != cudaSuccess ||
         cudaMalloc(&ctx->tick, sizeof(unsigned int) * (cfg->n_layers + 1)) != cudaSuccess ||
@@ -783,7 +904,16 @@ int faedkv_compress_prefill(faedkv_ctx *ctx, int layer, const void *K, const voi
     if (mode == FAEDKV_PREFILL_AUTO)
         mode = (c.kv_dtype == FAEDKV_BF16 && umma_prefill_available()) ? FAEDKV_PREFILL_UMMA : FAEDKV_PREFILL_SIMT;
     int r;
-    if (mode == FAEDKV_PREFILL_UMMA) {
+    if (ctx->prefill_fft) {
+        const int units = batch * c.n_kv_heads;
+        if (c.kv_dtype == FAEDKV_BF16) {
+            r = launch_prefill_fft_tensor<__nv_bfloat16>(ctx, *p, K, units, T, coefK, st);
+            if (r == 0) r = launch_prefill_fft_tensor<__nv_bfloat16>(ctx, *p, V, units, T, coefV, st);
+        } else {
+            r = launch_prefill_fft_tensor<float>(ctx, *p, K, units, T, coefK, st);
+            if (r == 0) r = launch_prefill_fft_tensor<float>(ctx, *p, V, units, T, coefV, st);
+        }
+    } else if (mode == FAEDKV_PREFILL_UMMA) {
         char msg[256] = {0};
         r = umma_prefill_launch(ctx->umma, K, V, batch, c.n_kv_heads, T, p->d_bins, p->M, c.n_dft,
                                 c.twiddle_terms == 2 ? 2 : 1, coefK, coefV, ctx->dev_status, st, msg, sizeof(msg));
@@ -834,6 +964,11 @@ int faedkv_reconstruct(faedkv_ctx *ctx, int layer, const float *coefK, const flo
     if (int r = check_ptrs(ctx, {coefK, coefV, K_out, V_out})) return r;
     if (int r = check_tlen(ctx, t_len)) return r;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->use_fft) {
+        if (ctx->cfg.kv_dtype == FAEDKV_BF16)
+            return launch_reconstruct_fft<__nv_bfloat16>(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);
+        return launch_reconstruct_fft<float>(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);
+    }
     if (ctx->use_tc) return launch_reconstruct_tc(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);
     if (ctx->cfg.kv_dtype == FAEDKV_BF16)
         return launch_reconstruct<__nv_bfloat16>(ctx, *p, coefK, coefV, t_len, batch, L, K_out, V_out, st);

@@ -1,0 +1,106 @@
+// FFT-shaped reconstruction (Eq. 11: Eq. 5 with every pruned bin zero) for power-of-two grids P:
+//
+//     x~[n, c] = (1/P) sum_k w_k (Re C[k,c] cos(w k n) - Im C[k,c] sin(w k n)),   n < min(t, P)
+//
+// as a real inverse FFT of the zero-filled half spectrum, per channel, with the two-pass scheme of
+// k_fft.cuh.  Columns are the channels of a run of consecutive (sequence, kv head) units of one tensor:
+// column = (unit - unit0) * 128 + c.
+//
+//   k_rfft_inv_a   gather the retained bins from the coefficient planes, pack the half spectrum,
+//                  pass A (over k1) + inter-pass twiddle                      -> Y [N1][N2][cols]
+//   k_rfft_inv_b   pass B (over k2); the complex result z[m] holds rows 2m and 2m+1, written in the
+//                  tensor's storage type; rows at or beyond the live length are written as zero
+#pragma once
+#include "common.cuh"
+#include "k_fft.cuh"
+
+namespace faedkv {
+
+// grid = (N2 / KT, cols / 16); block = 256; dynamic smem as k_afft_inv_a.
+// coef: planes of the tensor, [units][2][M][128]; unit0: first unit of this launch.
+template <int LG>
+__global__ void __launch_bounds__(fft::kThreads)
+k_rfft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float *__restrict__ coef, int M, int unit0,
+             float2 *__restrict__ Y, int lgKT) {
+    using namespace fft;
+    constexpr int NF = 1 << LG;                      // = N1
+    extern __shared__ float2 fft_smem[];
+    const int KT = 1 << lgKT, lg_cols = lgKT + kLgCW;
+    const int tile = NF << lg_cols;
+    float2 *xa = fft_smem, *xb = xa + (exchange_buffers(LG) > 0 ? tile : 0);
+    float2 *tw = xb + (exchange_buffers(LG) > 1 ? tile : 0);
+    float2 *tab_i = tw + NF;                         // [m1][kt]: e^{+j2pi k2 m1 / N}
+    float2 *tab_p = tab_i + (NF << lgKT);            // [k1][kt]: e^{+j2pi (N2 k1 + k2) / P}
+    const int k2_0 = blockIdx.x * KT, g0 = blockIdx.y * kCW;
+    fill_twiddles(tw, NF);
+    for (int e = threadIdx.x; e < (NF << lgKT); e += kThreads) {
+        const int kt = e & (KT - 1), r = e >> lgKT;
+        tab_i[e] = unit_phasor((uint32_t)((k2_0 + kt) * r), (uint32_t)g.N);
+        tab_p[e] = unit_phasor((uint32_t)(g.N2 * r + k2_0 + kt), g.P);
+    }
+    __syncthreads();
+    const float inv_P = 1.0f / (float)g.P;
+    const size_t plane = (size_t)M * kHeadDim;
+    auto load = [&](int k1, int cidx) {
+        const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
+        const int k = g.N2 * k1 + k2_0 + kt;                 // 0 <= k < N
+        const int col = g0 + c;
+        float2 z = make_float2(0.f, 0.f);
+        const int sa = slot[k], sb = slot[g.N - k];
+        if (sa >= 0 || sb >= 0) {
+            const float *u = coef + (size_t)(unit0 + (col >> 7)) * 2 * plane + (col & (kHeadDim - 1));
+            float2 xk = make_float2(0.f, 0.f), xm = make_float2(0.f, 0.f);
+            if (sa >= 0) xk = make_float2(u[(size_t)sa * kHeadDim], u[plane + (size_t)sa * kHeadDim]);
+            if (sb >= 0) xm = make_float2(u[(size_t)sb * kHeadDim], -u[plane + (size_t)sb * kHeadDim]);   // conj X[N-k]
+            if (k == 0) { xk.y = 0.f; xm.y = 0.f; }          // bins 0 and N = P/2 are their own mirrors
+            xk.x *= inv_P; xk.y *= inv_P; xm.x *= inv_P; xm.y *= inv_P;
+            z = cadd(cadd(xk, xm), cmulj(cmul(tab_p[(k1 << lgKT) + kt], csub(xk, xm))));
+        }
+        return z;
+    };
+    auto store = [&](int m1, int cidx, float2 v) {
+        const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
+        Y[y_index(g, m1, k2_0 + kt, g0 + c)] = cmul(v, tab_i[(m1 << lgKT) + kt]);
+    };
+    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+}
+
+// grid = (N1 / MT, cols / 16); block = 256; dynamic smem = rfft_smem_b(lgN2, lgMT).
+// out: rows of the tensor, [units][Lrows][128]; H: kv heads per sequence (t_len index = unit / H).
+template <int LG, typename TOut>
+__global__ void __launch_bounds__(fft::kThreads)
+k_rfft_inv_b(fft::Geometry g, const float2 *__restrict__ Y, const int32_t *__restrict__ t_len, int H, int unit0,
+             int Lrows, TOut *__restrict__ out, int lgMT) {
+    using namespace fft;
+    constexpr int NF = 1 << LG;                      // = N2
+    extern __shared__ float2 fft_smem[];
+    const int lg_cols = lgMT + kLgCW;
+    const int tile = NF << lg_cols;
+    float2 *xa = fft_smem, *xb = xa + (exchange_buffers(LG) > 0 ? tile : 0);
+    float2 *tw = xb + (exchange_buffers(LG) > 1 ? tile : 0);
+    const int m1_0 = blockIdx.x << lgMT, g0 = blockIdx.y * kCW;
+    fill_twiddles(tw, NF);
+    __syncthreads();
+    // the 16 columns of a CTA belong to one unit (128 channels per unit)
+    const int unit = unit0 + (g0 >> 7);
+    const int t = t_len[unit / H];
+    const int live = t < (int)g.P ? t : (int)g.P;
+    TOut *obase = out + (size_t)unit * Lrows * kHeadDim + (g0 & (kHeadDim - 1));
+    auto load = [&](int k2, int cidx) {
+        return Y[y_index(g, m1_0 + (cidx >> kLgCW), k2, g0 + (cidx & (kCW - 1)))];
+    };
+    auto store = [&](int m2, int cidx, float2 v) {
+        const int n = 2 * (m1_0 + (cidx >> kLgCW) + g.N1 * m2);
+        TOut *o = obase + (size_t)n * kHeadDim + (cidx & (kCW - 1));
+        if (n < Lrows) store1(o, n < live ? v.x : 0.f);
+        if (n + 1 < Lrows) store1(o + kHeadDim, n + 1 < live ? v.y : 0.f);
+    };
+    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+}
+
+inline size_t rfft_smem_b(int lg, int lgMT) {
+    const size_t nf = (size_t)1 << lg, tile = nf << (lgMT + fft::kLgCW);
+    return (fft::exchange_buffers(lg) * tile + nf) * sizeof(float2);
+}
+
+}  // namespace faedkv

@@ -81,6 +81,31 @@ def test_config1_full_prefill(fk, oracle):
     ctx.close()
 
 
+def test_config1_fft_prefill_layer(fk, oracle):
+    """configs[1], one layer through the FFT-shaped prefill: float32-exact coefficients from bf16 K/V."""
+    from helpers import REL_L2_F32
+    from paper_2507_20030_b200 import synth
+    H, HQ, T, M, l = 8, 32, 32768, 4096, 21
+    P = T
+    ctx = fk.Context(n_layers=l + 1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=1, kv_dtype=fk.BF16,
+                     prefill_mode=fk.PREFILL_FFT)
+    mask = fk.mask_mixed(P, M, l, synth.config_seed(1))
+    ctx.plan(l, mask)
+    bins = oracle.plan(P, mask)
+    K, V = synth.make_kv(synth.config_seed(1, l), 1, H, T, D, dtype=torch.bfloat16, device="cuda")
+    cK, cV = ctx.alloc_coef(l, 1), ctx.alloc_coef(l, 1)
+    t_len = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(l, K, V, cK, cV, t_len)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0 and t_len.tolist() == [T]
+    for h in (1, 6):
+        for x, c in ((K, cK), (V, cV)):
+            want = _oracle_unit_state(oracle, x[0, h].cpu(), P, bins, None, 0)
+            err = rel_l2(to_np64(c[0, h]), want)
+            assert err <= REL_L2_F32, (h, err)
+    ctx.close()
+
+
 def _decode_case(fk, oracle, *, config, layer, B, H, HQ, T, M, mask_kind, steps, sample_units, sample_steps,
                  coef_channels=None, fused_every=2):
     """Prefill one layer at full size, run `steps` decode steps (append + attention; every

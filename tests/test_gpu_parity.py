@@ -208,35 +208,41 @@ def test_checkpoint_restore_is_bit_exact(fk):
 # ----------------------------------------------------------------------------- reconstruct
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("P,M,L,B,H,tl", [(64, 33, 64, 2, 1, [64, 40]), (100, 20, 77, 1, 3, [300]),
-                                          (512, 100, 512, 1, 2, [512]), (96, 1, 50, 1, 1, [96])])
+                                          (512, 100, 512, 1, 2, [512]), (96, 1, 50, 1, 1, [96]),
+                                          (2048, 256, 2048, 1, 8, [2111]),      # config-0 shape after its 64 appends
+                                          (8192, 64, 5001, 2, 3, [8192, 77]),   # two-pass split 64 x 64; odd L; ragged
+                                          (256, 129, 255, 1, 1, [256])])        # every bin retained
 def test_reconstruct_matches_oracle(fk, oracle, dtype, P, M, L, B, H, tl):
-    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype))
     mask = _random_mask(P, M, 9 * P + L) if M > 1 else _mask_from_bins(P, [0])
-    ctx.plan(0, mask)
     bins = oracle.plan(P, mask)
     rng = np.random.default_rng(L)
     cK = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * P ** 0.5).astype(np.float32)).cuda()
     cV = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * P ** 0.5).astype(np.float32)).cuda()
     t_np = np.array(tl, dtype=np.int32)
     t_len = torch.from_numpy(t_np).cuda()
-    Ko = torch.full((B, H, L, 128), 7.0, dtype=dtype, device="cuda")
-    Vo = torch.full((B, H, L, 128), 7.0, dtype=dtype, device="cuda")
-    ctx.reconstruct(0, cK, cV, t_len, L, Ko, Vo)
-    torch.cuda.synchronize()
     wantK = oracle_reconstruct(oracle, to_np64(cK), P, bins, t_np, L)
     wantV = oracle_reconstruct(oracle, to_np64(cV), P, bins, t_np, L)
-    assert rel_l2(to_np64(Ko), wantK) <= _tol(dtype)
-    assert rel_l2(to_np64(Vo), wantV) <= _tol(dtype)
-    for b in range(B):                                           # rows past the live length are exactly zero
-        live = min(int(t_np[b]), P)
-        if live < L:
-            assert float(Ko[b, :, live:].abs().max()) == 0.0
-    # K only
-    Ko2 = torch.zeros_like(Ko)
-    ctx.reconstruct(0, cK, None, t_len, L, Ko2, None)
-    torch.cuda.synchronize()
-    assert torch.equal(Ko2, Ko)
-    ctx.close()
+    for mode in _decode_modes(fk, dtype, P):
+        ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                         decode_mode=mode)
+        ctx.plan(0, mask)
+        Ko = torch.full((B, H, L, 128), 7.0, dtype=dtype, device="cuda")
+        Vo = torch.full((B, H, L, 128), 7.0, dtype=dtype, device="cuda")
+        ctx.reconstruct(0, cK, cV, t_len, L, Ko, Vo)
+        torch.cuda.synchronize()
+        assert rel_l2(to_np64(Ko), wantK) <= _tol(dtype), mode
+        assert rel_l2(to_np64(Vo), wantV) <= _tol(dtype), mode
+        for b in range(B):                                           # rows past the live length are exactly zero
+            live = min(int(t_np[b]), P)
+            if live < L:
+                assert float(Ko[b, :, live:].abs().max()) == 0.0
+        # K only
+        Ko2 = torch.zeros_like(Ko)
+        ctx.reconstruct(0, cK, None, t_len, L, Ko2, None)
+        torch.cuda.synchronize()
+        assert torch.equal(Ko2, Ko)
+        assert ctx.device_status() == 0
+        ctx.close()
 
 
 def test_all_bins_round_trip(fk):
@@ -477,4 +483,37 @@ def test_prefill_umma_matches_oracle(fk, oracle, terms, tol, P, T, M, B, H):
     errK = rel_l2(to_np64(cK), oracle_compress(oracle, K, P, bins))
     errV = rel_l2(to_np64(cV), oracle_compress(oracle, V, P, bins))
     assert errK <= tol and errV <= tol, (errK, errV)
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- FFT-shaped prefill
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,T,M,B,H", [
+    (512, 512, 128, 1, 1),
+    (512, 300, 200, 1, 2),      # T < P: zero padding; odd split of the bins
+    (256, 1000, 129, 1, 2),     # T > P: positions wrap and add; every bin retained
+    (2048, 2048, 256, 1, 8),    # config-0 shape
+    (64, 1, 3, 1, 1),           # a single token on the smallest grid
+    (4096, 3001, 257, 2, 3),    # odd T (the last packed sample has no odd partner), several units per launch
+    (8192, 8192, 96, 1, 5),     # two-pass split 64 x 64
+])
+def test_prefill_fft_matches_oracle(fk, oracle, dtype, P, T, M, B, H):
+    """Float32-exact whatever the storage type: the FFT-shaped prefill meets the float32 bar on bf16 K/V too."""
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                     prefill_mode=fk.PREFILL_FFT)
+    mask = _random_mask(P, M, 11 * P + T)
+    mask[0] = 1
+    mask[P // 2] = 1                          # both self-conjugate bins
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    K, V = _make(41 + P + T, B, H, T, dtype)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    cK.fill_(float("nan")); cV.fill_(float("nan"))
+    t_len = torch.full((B,), -1, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0 and t_len.tolist() == [T] * B
+    errK = rel_l2(to_np64(cK), oracle_compress(oracle, K, P, bins))
+    errV = rel_l2(to_np64(cV), oracle_compress(oracle, V, P, bins))
+    assert errK <= REL_L2_F32 and errV <= REL_L2_F32, (errK, errV)
     ctx.close()
