@@ -12,6 +12,11 @@ masks keeping 1/8 of the bins):
        the fused faedkv_append_decode_attn                           -> decode us / layer / step
     C. faedkv_reconstruct of all 32 layers (L = P)
 
+Beside the timed step the line carries: `prefill_fft` (the same prefill through prefill_mode = FFT, the
+paper's own O(N log N) route, for comparison with the tensor-core contraction that `value` measures) and
+`decode.configs` (decode us / layer / step at the configs[2] and configs[3] shapes, whose state comes
+from a real prefill).
+
 Inputs are resident in HBM before the timed region; every layer's tensors are distinct and the layers
 are cycled (4 GiB of K/V, 2 GiB of coefficients), so nothing survives in the 126 MB L2 between uses.
 `e2e` repeats phase A through the same C-ABI calls with the K/V in pinned HOST memory and the
@@ -72,7 +77,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "200"],
+                 "--format=csv,noheader,nounits", "-lms", "100"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -178,7 +183,7 @@ DECODE_WORKLOADS = [
 ]
 
 
-def decode_section(torch, binding, synth, dev, W, peaks, iters):
+def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     """Decode us / layer / step at one workload shape: the state comes from a real prefill (one layer of
     K/V resident at a time), then the three decode calls are timed over all layers, each loop replayed
     as one CUDA graph (launch gaps excluded) and, for the fused call, also launched eagerly."""
@@ -220,6 +225,9 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters):
         b.record()
         torch.cuda.synchronize()
         eager_us = a.elapsed_time(b) / iters / NL * 1e3
+        if not graphs:
+            res[name] = {"us_eager_launches": eager_us}
+            continue
         graph = torch.cuda.CUDAGraph()
         side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(side):
@@ -240,8 +248,9 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters):
         gbs = alg_bytes[name] / (us * 1e-6) / 1e9
         res[name] = {"us": us, "us_eager_launches": eager_us, "bytes": alg_bytes[name], "bound": "hbm", "achieved": gbs,
                      "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"]}
-    res["decode_us_per_layer_step"] = res["append_decode_attn"]["us"]
-    res["decode_us_per_layer_step_two_calls"] = res["append"]["us"] + res["decode_attn"]["us"]
+    if graphs:
+        res["decode_us_per_layer_step"] = res["append_decode_attn"]["us"]
+        res["decode_us_per_layer_step_two_calls"] = res["append"]["us"] + res["decode_attn"]["us"]
     if ctx.device_status() != 0:
         raise RuntimeError("a kernel reported a device-side timeout; the numbers are invalid")
     ctx.close()
@@ -265,6 +274,17 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     build.build()
     peaks = _peaks()
+    if args.only_decode_config:
+        # small profiling case: one decode section alone, eager launches, optionally fewer layers
+        DW = dict(DECODE_WORKLOADS[args.only_decode_config - 2])
+        if args.layers:
+            DW["n_layers"] = args.layers
+            DW["name"] += f" [first {args.layers} layers only: profiling case, not a bench value]"
+        res = decode_section(torch, binding, synth, torch.device("cuda", local), DW, peaks, args.decode_config_iters,
+                             graphs=False)
+        if rank == 0:
+            print(json.dumps({"profiling_case": res}))
+        return
     W = dict(WORKLOAD)
     if args.layers:
         W["n_layers"] = args.layers
@@ -325,12 +345,12 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
+    sampler = ClockSampler(local)
+    for i in range(args.warmup):
+        if i == args.warmup - 1 and rank == 0:
+            sampler.start()          # nvidia-smi needs a moment to come up: start it one warm-up step early
         step(None)
     barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     launches0 = ctx.launch_count()
     rec = {}
     t_start, t_stop = ev(), ev()
@@ -415,6 +435,46 @@ def run_ours(args):
                "what": "phase A through the C ABI with pinned host K/V in and host coefficient planes out"}
         del hK, hV, hcK, hcV
 
+    # ---- the same prefill through the FFT-shaped path (comparison; not part of `value`)
+    prefill_fft = None
+    if not args.no_prefill_fft:
+        fctx = binding.Context(n_layers=NL, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=binding.BF16,
+                               prefill_mode=binding.PREFILL_FFT)
+        for l in range(NL):
+            fctx.plan(l, binding.mask_mixed(P, M, l, base_seed))
+
+        def fft_prefill():
+            for l in range(NL):
+                fctx.compress_prefill(l, Ks[l], Vs[l], cKs[l], cVs[l], tls[l])
+        fft_prefill()
+        barrier()
+        a, b = ev(), ev()
+        a.record(stream)
+        for _ in range(args.steps):
+            fft_prefill()
+        b.record(stream)
+        barrier()
+        f_ms = a.elapsed_time(b) / args.steps
+        if world > 1:
+            t = torch.tensor([f_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            f_ms = float(t[0])
+        n_cols = 2 * B * H * D                                           # channels of K and V
+        lgN = (P // 2).bit_length() - 1
+        flop = 5.0 * (P // 2) * lgN * n_cols                             # 5 N log2 N per complex length-N FFT
+        f_bytes = 2 * B * H * T * D * 2 + 2 * B * H * 2 * M * D * 4      # K/V in (bf16) + planes out (float32)
+        peak_alu = 148 * 128 * 2 * 1.965e9 / 1e12                        # float32 FMA lanes x 2 x max SM clock
+        prefill_fft = {"value": world * B * T / (f_ms * 1e-3), "unit": UNIT, "ms_per_layer": f_ms / NL,
+                       "speedup_vs_value_path": prefill_ms / f_ms, "precision": "float32 (rel. error ~1e-6)",
+                       "roofline": {"bound": "alu", "achieved": flop / (f_ms / NL * 1e-3) / 1e12, "peak": peak_alu,
+                                    "unit": "TFLOP/s", "frac": flop / (f_ms / NL * 1e-3) / 1e12 / peak_alu,
+                                    "flop_per_layer": flop, "flop_model": "5 N log2 N per channel, N = P/2",
+                                    "hbm_gbs": f_bytes / (f_ms / NL * 1e-3) / 1e9, "hbm_frac": f_bytes / (f_ms / NL * 1e-3) / 1e9 / peaks["hbm"],
+                                    "bytes_per_layer": f_bytes}}
+        if fctx.device_status() != 0:
+            raise RuntimeError("a kernel reported a device-side timeout; the numbers are invalid")
+        fctx.close()
+
     # ---- decode at the workloads that define it (streaming decode, long context)
     decode_sections = []
     if not args.no_decode_configs and not args.layers:
@@ -468,8 +528,11 @@ def run_ours(args):
         "decode_attn": {"us": attn_ms * 1e3, "bytes": coef_bytes, "bound": "hbm",
                         "achieved": coef_bytes / (attn_ms * 1e-3) / 1e9, "peak": peaks["hbm"], "unit": "GB/s",
                         "frac": coef_bytes / (attn_ms * 1e-3) / 1e9 / peaks["hbm"]},
-        "reconstruct": {"ms_per_layer": recon_ms, "flop": 2.0 * P * (2 * M) * n_c * 2,
-                        "achieved_tflops": 2.0 * P * (2 * M) * n_c * 2 / (recon_ms * 1e-3) / 1e12},
+        "reconstruct": {"us": recon_ms * 1e3, "bytes": coef_bytes + 2 * B * H * P * D * 2, "bound": "hbm",
+                        "achieved": (coef_bytes + 2 * B * H * P * D * 2) / (recon_ms * 1e-3) / 1e9, "peak": peaks["hbm"],
+                        "unit": "GB/s", "frac": (coef_bytes + 2 * B * H * P * D * 2) / (recon_ms * 1e-3) / 1e9 / peaks["hbm"],
+                        "what": "FFT-shaped (float32 two-pass FFT per channel); instruction-bound, bytes = planes in + bf16 rows out",
+                        "dense_equivalent_tflops": 2.0 * P * (2 * M) * n_c * 2 / (recon_ms * 1e-3) / 1e12},
         "decode_iters": n_dec,
     }
 
@@ -488,7 +551,7 @@ def run_ours(args):
                        "l2": "inputs larger than L2: 32 layers cycled, 128 MiB K/V + 64 MiB planes per layer",
                        "multi_gpu": "replicas only"},
             "phase_ms": phase_ms, "prefill_ms": prefill_ms,
-            "roofline": roofline, "decode": decode, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
+            "roofline": roofline, "prefill_fft": prefill_fft, "decode": decode, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
     print(json.dumps(line))
@@ -499,7 +562,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--decode-iters", type=int, default=2)
@@ -509,9 +572,13 @@ def main():
                     help="run only the first N layers of the workload (small case for profiler captures; "
                          "a bench value must use the default = all layers)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-prefill-fft", action="store_true", help="skip the FFT-shaped prefill comparison")
     ap.add_argument("--no-decode-configs", action="store_true",
                     help="skip the decode sections at the configs[2] and configs[3] shapes")
     ap.add_argument("--decode-config-iters", type=int, default=10)
+    ap.add_argument("--only-decode-config", type=int, default=0, choices=[0, 2, 3],
+                    help="profiling case: run only the decode section of configs[2] or configs[3] (eager launches; "
+                         "combine with --layers and --decode-config-iters 1)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
