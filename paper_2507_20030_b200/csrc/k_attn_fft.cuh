@@ -101,23 +101,24 @@ k_afft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float2 *__
     float2 *tw = xb + (exchange_buffers(LG) > 1 ? tile : 0);
     float2 *tab_i = tw + NF;                         // [m1][kt]: e^{+j2pi k2 m1 / N}
     float2 *tab_p = tab_i + (NF << lgKT);            // [k1][kt]: e^{+j2pi (N2 k1 + k2) / P}
+    int2 *tab_s = reinterpret_cast<int2 *>(tab_p + (NF << lgKT));   // [k1][kt]: plan slots of bins k and N - k (or -1)
     const int k2_0 = blockIdx.x * KT, g0 = blockIdx.y * kCW;
     fill_twiddles(tw, NF);
     for (int e = threadIdx.x; e < (NF << lgKT); e += kThreads) {
         const int kt = e & (KT - 1), r = e >> lgKT;
         tab_i[e] = unit_phasor((uint32_t)((k2_0 + kt) * r), (uint32_t)g.N);      // k2 * m1 < N2 * N1 = N
         tab_p[e] = unit_phasor((uint32_t)(g.N2 * r + k2_0 + kt), g.P);
+        tab_s[e] = make_int2(slot[g.N2 * r + k2_0 + kt], slot[g.N - (g.N2 * r + k2_0 + kt)]);
     }
     __syncthreads();
     auto load = [&](int k1, int cidx) {
         const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
-        const int k = g.N2 * k1 + k2_0 + kt;                 // 0 <= k < N
         const int col = g0 + c;
         float2 z = make_float2(0.f, 0.f);
-        const int sa = slot[k], sb = slot[g.N - k];
-        if ((sa >= 0 || sb >= 0) && col < g.G) {
-            const float2 xk = sa >= 0 ? Qs[(uint32_t)sa * (uint32_t)g.Gp + (uint32_t)col] : make_float2(0.f, 0.f);
-            float2 xm = sb >= 0 ? Qs[(uint32_t)sb * (uint32_t)g.Gp + (uint32_t)col] : make_float2(0.f, 0.f);
+        const int2 sl = tab_s[(k1 << lgKT) + kt];
+        if ((sl.x >= 0 || sl.y >= 0) && col < g.G) {
+            const float2 xk = sl.x >= 0 ? Qs[(uint32_t)sl.x * (uint32_t)g.Gp + (uint32_t)col] : make_float2(0.f, 0.f);
+            float2 xm = sl.y >= 0 ? Qs[(uint32_t)sl.y * (uint32_t)g.Gp + (uint32_t)col] : make_float2(0.f, 0.f);
             xm.y = -xm.y;                                            // conj X[N-k]
             z = cadd(cadd(xk, xm), cmulj(cmul(tab_p[(k1 << lgKT) + kt], csub(xk, xm))));
         }
@@ -295,7 +296,8 @@ k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restr
 // Dynamic shared memory of the three kernels above (bytes).
 inline size_t afft_smem_a(int lg, int lgKT, bool packing_table) {
     const size_t nf = (size_t)1 << lg, tile = nf << (lgKT + fft::kLgCW);
-    return (fft::exchange_buffers(lg) * tile + nf + (packing_table ? 2 : 1) * (nf << lgKT)) * sizeof(float2);
+    // exchange buffers, twiddles, inter-pass twiddles (+ packing phasors and slot pairs)
+    return (fft::exchange_buffers(lg) * tile + nf + (packing_table ? 3 : 1) * (nf << lgKT)) * sizeof(float2);
 }
 inline size_t afft_smem_mid(int lg, int lgMT) {
     const size_t nf = (size_t)1 << lg, tile = nf << (lgMT + fft::kLgCW);

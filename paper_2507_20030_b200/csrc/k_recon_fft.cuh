@@ -31,28 +31,29 @@ k_rfft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float *__r
     float2 *tw = xb + (exchange_buffers(LG) > 1 ? tile : 0);
     float2 *tab_i = tw + NF;                         // [m1][kt]: e^{+j2pi k2 m1 / N}
     float2 *tab_p = tab_i + (NF << lgKT);            // [k1][kt]: e^{+j2pi (N2 k1 + k2) / P}
+    int2 *tab_s = reinterpret_cast<int2 *>(tab_p + (NF << lgKT));   // [k1][kt]: plan slots of bins k and N - k (or -1)
     const int k2_0 = blockIdx.x * KT, g0 = blockIdx.y * kCW;
     fill_twiddles(tw, NF);
     for (int e = threadIdx.x; e < (NF << lgKT); e += kThreads) {
         const int kt = e & (KT - 1), r = e >> lgKT;
         tab_i[e] = unit_phasor((uint32_t)((k2_0 + kt) * r), (uint32_t)g.N);
         tab_p[e] = unit_phasor((uint32_t)(g.N2 * r + k2_0 + kt), g.P);
+        tab_s[e] = make_int2(slot[g.N2 * r + k2_0 + kt], slot[g.N - (g.N2 * r + k2_0 + kt)]);
     }
     __syncthreads();
     const float inv_P = 1.0f / (float)g.P;
     const size_t plane = (size_t)M * kHeadDim;
     auto load = [&](int k1, int cidx) {
         const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
-        const int k = g.N2 * k1 + k2_0 + kt;                 // 0 <= k < N
         const int col = g0 + c;
         float2 z = make_float2(0.f, 0.f);
-        const int sa = slot[k], sb = slot[g.N - k];
-        if (sa >= 0 || sb >= 0) {
+        const int2 sl = tab_s[(k1 << lgKT) + kt];
+        if (sl.x >= 0 || sl.y >= 0) {
             const float *u = coef + (size_t)(unit0 + (col >> 7)) * 2 * plane + (col & (kHeadDim - 1));
             float2 xk = make_float2(0.f, 0.f), xm = make_float2(0.f, 0.f);
-            if (sa >= 0) xk = make_float2(u[(size_t)sa * kHeadDim], u[plane + (size_t)sa * kHeadDim]);
-            if (sb >= 0) xm = make_float2(u[(size_t)sb * kHeadDim], -u[plane + (size_t)sb * kHeadDim]);   // conj X[N-k]
-            if (k == 0) { xk.y = 0.f; xm.y = 0.f; }          // bins 0 and N = P/2 are their own mirrors
+            if (sl.x >= 0) xk = make_float2(u[(uint32_t)sl.x * kHeadDim], u[plane + (uint32_t)sl.x * kHeadDim]);
+            if (sl.y >= 0) xm = make_float2(u[(uint32_t)sl.y * kHeadDim], -u[plane + (uint32_t)sl.y * kHeadDim]);   // conj X[N-k]
+            if (k1 == 0 && k2_0 + kt == 0) { xk.y = 0.f; xm.y = 0.f; }   // k = 0: bins 0 and N = P/2 are their own mirrors
             xk.x *= inv_P; xk.y *= inv_P; xm.x *= inv_P; xm.y *= inv_P;
             z = cadd(cadd(xk, xm), cmulj(cmul(tab_p[(k1 << lgKT) + kt], csub(xk, xm))));
         }
@@ -91,7 +92,7 @@ k_rfft_inv_b(fft::Geometry g, const float2 *__restrict__ Y, const int32_t *__res
     };
     auto store = [&](int m2, int cidx, float2 v) {
         const int n = 2 * (m1_0 + (cidx >> kLgCW) + g.N1 * m2);
-        TOut *o = obase + (size_t)n * kHeadDim + (cidx & (kCW - 1));
+        TOut *o = obase + (uint32_t)n * (uint32_t)kHeadDim + (uint32_t)(cidx & (kCW - 1));   // n < P <= 2^19
         if (n < Lrows) store1(o, n < live ? v.x : 0.f);
         if (n + 1 < Lrows) store1(o + kHeadDim, n + 1 < live ? v.y : 0.f);
     };
