@@ -92,6 +92,10 @@ typedef struct {
                           (rel. error ~1e-3), 2 = bf16 hi+lo pair (~1e-5, twice the
                           MMA work); 0 = default (1)                                */
     int decode_mode;   /* faedkv_decode_mode                                       */
+    int n_sink;        /* S >= 0: first tokens kept in the time domain (Sec. 4.2; the paper
+                          uses 10).  Only the *_windowed calls look at n_sink / n_recent */
+    int n_recent;      /* R >= 0: most recent tokens kept in the time domain (the paper
+                          uses 50); n_sink + n_recent <= 1024                        */
 } faedkv_config;
 
 /* Create a context on the CURRENT CUDA device.  Allocates the scratch area
@@ -180,6 +184,41 @@ int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *c
 int faedkv_append_decode_attn(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new,
                               const void *q, int batch, float *coefK, float *coefV, int32_t *t_len,
                               float scale, void *out, void *stream);
+
+/* ---- sink and recent window (Sec. 4.2; Eq. 10, 12, 13) -------------------------------------------
+ * The paper's own workflow keeps the first S = n_sink tokens and the last R = n_recent tokens of a
+ * sequence in the time domain; only the tokens between them live in the frequency domain.  A
+ * window tensor (one for K, one for V; caller-owned, kv_dtype) has the layout
+ *   [batch][n_kv_heads][S + R][head_dim]:  rows [0, S) the sink tokens, rows [S, S + R) a ring in
+ *   which token n >= S occupies slot (n - S) mod R while it is among the last R tokens.
+ * t_len counts ALL tokens of a sequence; the transformed segment holds t_len - S - R of them, at
+ * positions 0, 1, ... (token n sits at position n - S), wrapping modulo P like everywhere else. */
+
+/* Bytes of ONE window tensor (K or V) at this batch. */
+size_t faedkv_window_bytes(const faedkv_ctx *ctx, int batch);
+
+/* Prefill (Eq. 10): tokens [0, S) are copied to the sink rows, tokens [T - R, T) to their ring
+ * slots, and the tokens between them are transformed into coefK, coefV as in
+ * faedkv_compress_prefill (planes are zero when there is none).  SETS t_len[b] = T.
+ * T >= S + R is required (FAEDKV_ERR_SHAPE otherwise).  With S = R = 0 this is
+ * faedkv_compress_prefill and winK, winV may be NULL. */
+int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch,
+                            int T, float *coefK, float *coefV, void *winK, void *winV,
+                            int32_t *t_len, void *stream);
+
+/* One decode step of the paper's workflow for every sequence, t = t_len[b]:
+ *   update (Eq. 12)  the token leaving the recent window, t - R, is folded into the coefficients
+ *                    at position t - R - S with unit weight (with R = 0: the new token itself);
+ *   attend (Eq. 13, Eq. 3)  out = softmax(scale * q . [K_sink | K~ | K_recent]) [V_sink | V~ | V_recent]
+ *                    over the S sink tokens, the reconstruction of min(t + 1 - S - R, P) positions
+ *                    and the R most recent tokens including the new one -- one softmax, evaluated
+ *                    without writing K~, V~ or the scores to memory;
+ *   commit           the new token takes the ring slot of the one that left; t_len[b] += 1.
+ * Needs the FFT-shaped decode path (P a power of two in [64, 2^19]); FAEDKV_ERR_UNSUPPORTED
+ * otherwise.  winK, winV, coefK, coefV and t_len are updated in place. */
+int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new,
+                         const void *q, int batch, float *coefK, float *coefV, void *winK,
+                         void *winV, int32_t *t_len, float scale, void *out, void *stream);
 
 /* Device-side status word of the context (host read; synchronises `stream`):
  * 0, or a nonzero code left by a kernel whose bounded wait on an mbarrier gave

@@ -220,3 +220,66 @@ def running_mean_step(Sre, Sim, P, bins, t, xnew):
     bins = np.ascontiguousarray(bins, dtype=np.int32)
     M, d = Sre.shape
     _load().orc_running_mean_step(_d(Sre), _d(Sim), M, d, P, _i(bins), t, _d(_f64arr(xnew)))
+
+
+# ---------------------------------------------------------------------------------------------------
+# Sink and recent window (Sec. 4.2): the paper's own decode workflow for ONE (sequence, kv head) unit,
+# written as a composition of the primitives above -- no new arithmetic.
+class WindowedUnit:
+    """State of one unit: the first S tokens (sink) and the last R tokens (recent) in the time domain,
+    the tokens between them as retained DFT coefficients of the segment that starts at token S."""
+
+    def __init__(self, P: int, bins: np.ndarray, S: int, R: int):
+        self.P, self.bins, self.S, self.R = int(P), np.ascontiguousarray(bins, dtype=np.int32), int(S), int(R)
+        self.t = 0
+        self.sinkK = self.sinkV = None
+        self.recentK, self.recentV = [], []          # oldest first
+        self.CK = self.CV = None                     # (re, im) pairs of [M, d]
+
+    def prefill(self, K: np.ndarray, V: np.ndarray) -> None:
+        """Eq. 10: transform K[S : T-R], V[S : T-R]; keep the first S and last R rows as they are."""
+        K, V = _f64arr(K), _f64arr(V)
+        T, d = K.shape
+        S, R = self.S, self.R
+        assert T >= S + R
+        self.sinkK, self.sinkV = K[:S].copy(), V[:S].copy()
+        self.recentK = [K[n].copy() for n in range(T - R, T)]
+        self.recentV = [V[n].copy() for n in range(T - R, T)]
+        M = self.bins.shape[0]
+        if T - S - R > 0:
+            self.CK = [np.ascontiguousarray(a) for a in compress(K[S:T - R], self.P, self.bins)]
+            self.CV = [np.ascontiguousarray(a) for a in compress(V[S:T - R], self.P, self.bins)]
+        else:
+            self.CK = [np.zeros((M, d)), np.zeros((M, d))]
+            self.CV = [np.zeros((M, d)), np.zeros((M, d))]
+        self.t = T
+
+    def step(self, k_new: np.ndarray, v_new: np.ndarray) -> None:
+        """Eq. 12: the token leaving the recent window is folded at the next position of the transformed
+        segment; the new token enters the window.  With R = 0 the new token itself is folded."""
+        k_new, v_new = _f64arr(k_new), _f64arr(v_new)
+        pos = self.t - self.S - self.R                # tokens already in the transformed segment
+        self.recentK.append(k_new.copy())
+        self.recentV.append(v_new.copy())
+        k_old, v_old = self.recentK.pop(0), self.recentV.pop(0)
+        append(self.CK[0], self.CK[1], self.P, self.bins, pos, k_old)
+        append(self.CV[0], self.CV[1], self.P, self.bins, pos, v_old)
+        self.t += 1
+
+    def attention(self, q: np.ndarray, scale: float | None = None) -> np.ndarray:
+        """Eq. 13 then Eq. 3: one softmax over [sink | reconstructed segment | recent]."""
+        q = _f64arr(q)
+        d = q.shape[1]
+        if scale is None:
+            scale = 1.0 / np.sqrt(d)
+        L = min(self.t - self.S - self.R, self.P)
+        parts_k, parts_v = [self.sinkK], [self.sinkV]
+        if L > 0:
+            parts_k.append(reconstruct(self.CK[0], self.CK[1], self.P, self.bins, L))
+            parts_v.append(reconstruct(self.CV[0], self.CV[1], self.P, self.bins, L))
+        if self.R > 0:
+            parts_k.append(np.stack(self.recentK))
+            parts_v.append(np.stack(self.recentV))
+        Kt = np.concatenate([p for p in parts_k if p.shape[0] > 0], axis=0)
+        Vt = np.concatenate([p for p in parts_v if p.shape[0] > 0], axis=0)
+        return attention_dense(q, Kt, Vt, scale)

@@ -27,7 +27,8 @@ EXPORTS = [
     "faedkv_create", "faedkv_destroy", "faedkv_last_error", "faedkv_plan", "faedkv_n_bins",
     "faedkv_get_bins", "faedkv_coef_bytes", "faedkv_mask_lowpass", "faedkv_mask_mixed",
     "faedkv_compress_prefill", "faedkv_append", "faedkv_reconstruct", "faedkv_decode_attn",
-    "faedkv_append_decode_attn", "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
+    "faedkv_append_decode_attn", "faedkv_window_bytes", "faedkv_prefill_windowed", "faedkv_step_windowed",
+    "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -42,7 +43,7 @@ class FaedkvError(RuntimeError):
 class Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "n_layers", "n_kv_heads", "n_q_heads", "head_dim", "n_dft", "max_batch", "kv_dtype",
-        "prefill_mode", "twiddle_terms", "decode_mode")]
+        "prefill_mode", "twiddle_terms", "decode_mode", "n_sink", "n_recent")]
 
 
 _lib = None
@@ -88,6 +89,12 @@ def load() -> ctypes.CDLL:
     lib.faedkv_decode_attn.restype = _int
     lib.faedkv_append_decode_attn.argtypes = [_vp, _int, _vp, _vp, _vp, _int, _vp, _vp, _vp, ctypes.c_float, _vp, _vp]
     lib.faedkv_append_decode_attn.restype = _int
+    lib.faedkv_window_bytes.argtypes = [_vp, _int]
+    lib.faedkv_window_bytes.restype = ctypes.c_size_t
+    lib.faedkv_prefill_windowed.argtypes = [_vp, _int, _vp, _vp, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp]
+    lib.faedkv_prefill_windowed.restype = _int
+    lib.faedkv_step_windowed.argtypes = [_vp, _int, _vp, _vp, _vp, _int, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp]
+    lib.faedkv_step_windowed.restype = _int
     lib.faedkv_device_status.argtypes = [_vp, _vp]
     lib.faedkv_device_status.restype = _int
     lib.faedkv_decode_attn_static.argtypes = [_int, _int, _int, _int, _vp, _int, _vp, _vp, _vp, _vp, _int,
@@ -162,11 +169,14 @@ class Context:
     prefill_mode: int = PREFILL_AUTO
     twiddle_terms: int = 0
     decode_mode: int = DECODE_AUTO
+    n_sink: int = 0
+    n_recent: int = 0
 
     def __post_init__(self):
         self._lib = load()
         cfg = Config(self.n_layers, self.n_kv_heads, self.n_q_heads, self.head_dim, self.n_dft,
-                     self.max_batch, self.kv_dtype, self.prefill_mode, self.twiddle_terms, self.decode_mode)
+                     self.max_batch, self.kv_dtype, self.prefill_mode, self.twiddle_terms, self.decode_mode,
+                     self.n_sink, self.n_recent)
         h = _vp()
         rc = self._lib.faedkv_create(ctypes.byref(cfg), ctypes.byref(h))
         if rc != 0:
@@ -251,6 +261,24 @@ class Context:
         self._check(self._lib.faedkv_append_decode_attn(
             self._h, layer, _ptr(k_new), _ptr(v_new), _ptr(q), batch, _ptr(coefK), _ptr(coefV), _ptr(t_len),
             float(scale), _ptr(out), _stream(stream)))
+
+    # -- sink + recent window
+    def alloc_window(self, batch: int, device="cuda") -> torch.Tensor:
+        """[batch, n_kv_heads, n_sink + n_recent, head_dim] in the storage type (uninitialised)."""
+        return torch.empty((batch, self.n_kv_heads, self.n_sink + self.n_recent, self.head_dim),
+                           dtype=self.torch_dtype, device=device)
+
+    def prefill_windowed(self, layer, K, V, coefK, coefV, winK, winV, t_len, stream=None):
+        batch, T = K.shape[0], K.shape[2]
+        self._check(self._lib.faedkv_prefill_windowed(
+            self._h, layer, _ptr(K), _ptr(V), batch, T, _ptr(coefK), _ptr(coefV), _ptr(winK), _ptr(winV),
+            _ptr(t_len), _stream(stream)))
+
+    def step_windowed(self, layer, k_new, v_new, q, coefK, coefV, winK, winV, t_len, out, scale: float = 0.0, stream=None):
+        batch = q.shape[0]
+        self._check(self._lib.faedkv_step_windowed(
+            self._h, layer, _ptr(k_new), _ptr(v_new), _ptr(q), batch, _ptr(coefK), _ptr(coefV), _ptr(winK),
+            _ptr(winV), _ptr(t_len), float(scale), _ptr(out), _stream(stream)))
 
     def launch_count(self) -> int:
         return int(self._lib.faedkv_launch_count(self._h))

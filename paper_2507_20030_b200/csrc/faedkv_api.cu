@@ -46,7 +46,8 @@ struct FftScratch {
     float2 *Yr = nullptr;                 // two-pass array of the FFT-shaped reconstruction / prefill, [N][recon_units * 128]
     float2 *Zr = nullptr;                 // second array of the FFT-shaped prefill (full spectrum before the gather)
     int recon_units = 0;                  // units (sequence, kv head) per launch group of the reconstruction
-    float *mloc = nullptr, *sloc = nullptr, *colsum = nullptr;
+    float *mloc = nullptr, *sloc = nullptr, *colsum = nullptr;   // [N1 + 1][Gp] (last row: the window), [2][Gp]
+    float *o_win = nullptr;               // [Gp][128] unnormalised attention output over the sink + recent window
     unsigned int *tickets = nullptr;      // [max_batch * H + max_batch], zero between calls
     int max_M = 0;
     unsigned int attr_mask[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
@@ -154,7 +155,7 @@ void free_scratch(faedkv_ctx *ctx) {
     cudaFree(t.cmax); cudaFree(t.psum); cudaFree(t.colsum); cudaFree(t.PfS);
     t = TcScratch();
     FftScratch &f = ctx->fs;
-    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr);
+    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.o_win); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr);
     f = FftScratch();
 }
 
@@ -189,9 +190,10 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
         if (f.Y == nullptr) {
             CUDA_TRY(ctx, cudaMalloc(&f.Y, (size_t)g.N * g.Gp * sizeof(float2)));
             CUDA_TRY(ctx, cudaMalloc(&f.Zf, (size_t)g.N * g.Gp * sizeof(float2)));
-            CUDA_TRY(ctx, cudaMalloc(&f.mloc, (size_t)g.N1 * g.Gp * sizeof(float)));
-            CUDA_TRY(ctx, cudaMalloc(&f.sloc, (size_t)g.N1 * g.Gp * sizeof(float)));
-            CUDA_TRY(ctx, cudaMalloc(&f.colsum, (size_t)g.Gp * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&f.mloc, (size_t)(g.N1 + 1) * g.Gp * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&f.sloc, (size_t)(g.N1 + 1) * g.Gp * sizeof(float)));
+            CUDA_TRY(ctx, cudaMalloc(&f.colsum, (size_t)2 * g.Gp * sizeof(float)));
+            if (c.n_sink + c.n_recent > 0) CUDA_TRY(ctx, cudaMalloc(&f.o_win, (size_t)g.Gp * kHeadDim * sizeof(float)));
             const size_t n_tickets = (size_t)c.max_batch * c.n_kv_heads + c.max_batch;
             CUDA_TRY(ctx, cudaMalloc(&f.tickets, n_tickets * sizeof(unsigned int)));
             CUDA_TRY(ctx, cudaMemset(f.tickets, 0, n_tickets * sizeof(unsigned int)));
@@ -475,7 +477,7 @@ int launch_reconstruct_fft(faedkv_ctx *ctx, const LayerPlan &p, const float *coe
 
 // FFT-shaped prefill of one tensor: (pass A', pass B', gather) over runs of units.
 template <typename TIn>
-int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x, int units, int T, float *coef,
+int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x, int units, int T, int T_stride, float *coef,
                               cudaStream_t st) {
     const faedkv_config &c = ctx->cfg;
     FftScratch &f = ctx->fs;
@@ -493,7 +495,7 @@ int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x
             const size_t smem = pfft_smem_a(g.lgN2, lgMT);
 #define CALL(LG)                                                                                         \
             rc = fft_opt_in(ctx, k_pfft_fwd_a<LG, TIn>, smem, f.attr_mask[kInKind], LG);                 \
-            if (rc == 0) k_pfft_fwd_a<LG, TIn><<<grid, fft::kThreads, smem, st>>>(g, static_cast<const TIn *>(x), T, u0, f.Yr, lgMT)
+            if (rc == 0) k_pfft_fwd_a<LG, TIn><<<grid, fft::kThreads, smem, st>>>(g, static_cast<const TIn *>(x), T, T_stride, u0, f.Yr, lgMT)
             FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
 #undef CALL
             if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
@@ -522,11 +524,20 @@ int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x
 
 // FFT-shaped decode attention; with APPEND the IWDFT update of K and V rides on the two coefficient
 // streams and the token counters advance at the end.
+// A windowed step (winK != nullptr) folds the token leaving the recent ring instead of the new one, lets the
+// sink + recent tokens join the softmax as one more tile, and ends by committing the new token to the ring.
 template <typename TQ, int GQ, bool APPEND>
 int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const void *k_new, const void *v_new,
-                    float *coefK, float *coefV, int32_t *t_len, int batch, float scale, void *out, cudaStream_t st) {
+                    float *coefK, float *coefV, int32_t *t_len, int batch, float scale, void *out, cudaStream_t st,
+                    void *winK = nullptr, void *winV = nullptr) {
     const faedkv_config &c = ctx->cfg;
     FftScratch &f = ctx->fs;
+    const bool windowed = winK != nullptr;
+    const int S = windowed ? c.n_sink : 0, R = windowed ? c.n_recent : 0;
+    const int n_extra = (windowed && S + R > 0) ? 1 : 0;
+    // the folded token: the call's new token, or with a ring the token that leaves it
+    const FoldSrc fold{(windowed && R > 0) ? S + R : 1, S, R};
+    const void *foldK = (windowed && R > 0) ? winK : k_new, *foldV = (windowed && R > 0) ? winV : v_new;
     const int H = c.n_kv_heads, HQ = c.n_q_heads, M = p.M, P = c.n_dft;
     const fft::Geometry g = fft::make_geometry(P, batch * HQ);
     const int col_blocks = g.Gp / fft::kCW;
@@ -536,9 +547,17 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
     {
         dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
         k_attn_qs<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(static_cast<const TQ *>(q), coefK,
-                                                                     static_cast<const TQ *>(k_new), t_len, p.d_bins, f.Qs, M, H,
-                                                                     HQ, g.Gp, (uint32_t)P, scale / (float)P);
+                                                                     static_cast<const TQ *>(foldK), t_len, p.d_bins, f.Qs, M, H,
+                                                                     HQ, g.Gp, (uint32_t)P, scale / (float)P, fold);
         if (int r = launch_check(ctx, "k_attn_qs")) return r;
+    }
+    if (n_extra) {
+        const int n_tiles = g.N1 >> lgMT;
+        k_attn_window<TQ, GQ><<<batch * H, 256, (size_t)GQ * (S + R) * sizeof(float), st>>>(
+            static_cast<const TQ *>(q), static_cast<const TQ *>(winK), static_cast<const TQ *>(winV),
+            static_cast<const TQ *>(k_new), static_cast<const TQ *>(v_new), t_len, H, S, R, scale,
+            f.mloc + (size_t)n_tiles * g.Gp, f.sloc + (size_t)n_tiles * g.Gp, f.o_win);
+        if (int r = launch_check(ctx, "k_attn_window")) return r;
     }
     int rc = FAEDKV_ERR_UNSUPPORTED;
     {
@@ -558,7 +577,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const size_t smem = afft_smem_mid(g.lgN2, lgMT);
 #define CALL(LG)                                                                                         \
         rc = fft_opt_in(ctx, k_afft_mid<LG>, smem, f.attr_mask[1], LG);                                  \
-        if (rc == 0) k_afft_mid<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Y, t_len, HQ, APPEND ? 1 : 0, f.mloc, f.sloc, lgMT)
+        if (rc == 0) k_afft_mid<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Y, t_len, HQ, (APPEND ? 1 : 0) - S - R, f.mloc, f.sloc, lgMT)
         FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
@@ -570,7 +589,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const size_t smem = afft_smem_fwd_b(g.lgN1, lgKT, lgMT);
 #define CALL(LG)                                                                                         \
         rc = fft_opt_in(ctx, k_afft_fwd_b<LG>, smem, f.attr_mask[2], LG);                                \
-        if (rc == 0) k_afft_fwd_b<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Y, f.mloc, f.sloc, lgMT, f.Zf, f.colsum, lgKT)
+        if (rc == 0) k_afft_fwd_b<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Y, f.mloc, f.sloc, lgMT, f.Zf, f.colsum, lgKT, n_extra)
         FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
@@ -581,21 +600,27 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const int per = (M + slices - 1) / slices;
         dim3 grid(slices, batch * H);
         k_attn_out_fft<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(
-            coefV, static_cast<const TQ *>(v_new), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
-            static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P);
+            coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
+            static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, windowed ? 0 : 1);
         if (int r = launch_check(ctx, "k_attn_out_fft")) return r;
+    }
+    if (windowed) {
+        k_window_commit<TQ><<<batch, kHeadDim, 0, st>>>(static_cast<const TQ *>(k_new), static_cast<const TQ *>(v_new),
+                                                        static_cast<TQ *>(winK), static_cast<TQ *>(winV), t_len, H, S, R);
+        if (int r = launch_check(ctx, "k_window_commit")) return r;
     }
     return FAEDKV_OK;
 }
 
 template <typename TQ, bool APPEND>
 int dispatch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const void *k_new, const void *v_new,
-                      float *coefK, float *coefV, int32_t *t_len, int batch, float scale, void *out, cudaStream_t st) {
+                      float *coefK, float *coefV, int32_t *t_len, int batch, float scale, void *out, cudaStream_t st,
+                      void *winK = nullptr, void *winV = nullptr) {
     switch (ctx->gq) {
-        case 1: return launch_attn_fft<TQ, 1, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
-        case 2: return launch_attn_fft<TQ, 2, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
-        case 4: return launch_attn_fft<TQ, 4, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
-        case 8: return launch_attn_fft<TQ, 8, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
+        case 1: return launch_attn_fft<TQ, 1, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+        case 2: return launch_attn_fft<TQ, 2, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+        case 4: return launch_attn_fft<TQ, 4, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+        case 8: return launch_attn_fft<TQ, 8, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
     }
     return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be 1, 2, 4 or 8");
 }
@@ -607,12 +632,12 @@ __global__ void k_set_tlen(int32_t *t_len, int batch, int T) {
 
 template <typename TIn>
 int launch_prefill_simt(faedkv_ctx *ctx, const LayerPlan &p, const void *K, const void *V, int batch,
-                        int T, float *coefK, float *coefV, cudaStream_t st) {
+                        int T, int T_stride, float *coefK, float *coefV, cudaStream_t st) {
     const faedkv_config &c = ctx->cfg;
     DftUnitArgs a{};
     a.x[0] = K; a.x[1] = V;
     a.y[0] = coefK; a.y[1] = coefV;
-    a.x_unit = (long long)T * kHeadDim;
+    a.x_unit = (long long)T_stride * kHeadDim;
     a.y_unit = 2LL * p.M * kHeadDim;
     a.y_plane = (long long)p.M * kHeadDim;
     a.x_row = kHeadDim; a.y_row = kHeadDim; a.col_blocks = 1;
@@ -696,6 +721,35 @@ int launch_attn(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const float 
     return FAEDKV_OK;
 }
 
+// The prefill transform of rows [0, T) of every unit of K and V (units T_stride rows apart) into the planes,
+// by whichever evaluation the context was configured for.
+int prefill_core(faedkv_ctx *ctx, const LayerPlan &p, const void *K, const void *V, int batch, int T, int T_stride,
+                 float *coefK, float *coefV, cudaStream_t st) {
+    const faedkv_config &c = ctx->cfg;
+    int mode = c.prefill_mode;
+    if (mode == FAEDKV_PREFILL_AUTO)
+        mode = (c.kv_dtype == FAEDKV_BF16 && umma_prefill_available()) ? FAEDKV_PREFILL_UMMA : FAEDKV_PREFILL_SIMT;
+    if (ctx->prefill_fft) {
+        const int units = batch * c.n_kv_heads;
+        if (c.kv_dtype == FAEDKV_BF16) {
+            if (int r = launch_prefill_fft_tensor<__nv_bfloat16>(ctx, p, K, units, T, T_stride, coefK, st)) return r;
+            return launch_prefill_fft_tensor<__nv_bfloat16>(ctx, p, V, units, T, T_stride, coefV, st);
+        }
+        if (int r = launch_prefill_fft_tensor<float>(ctx, p, K, units, T, T_stride, coefK, st)) return r;
+        return launch_prefill_fft_tensor<float>(ctx, p, V, units, T, T_stride, coefV, st);
+    }
+    if (mode == FAEDKV_PREFILL_UMMA) {
+        char msg[256] = {0};
+        int r = umma_prefill_launch(ctx->umma, K, V, batch, c.n_kv_heads, T, T_stride, p.d_bins, p.M, c.n_dft,
+                                    c.twiddle_terms == 2 ? 2 : 1, coefK, coefV, ctx->dev_status, st, msg, sizeof(msg));
+        if (r != 0) return fail(ctx, r, "%s", msg);
+        ctx->launches += 1;
+        return FAEDKV_OK;
+    }
+    if (c.kv_dtype == FAEDKV_BF16) return launch_prefill_simt<__nv_bfloat16>(ctx, p, K, V, batch, T, T_stride, coefK, coefV, st);
+    return launch_prefill_simt<float>(ctx, p, K, V, batch, T, T_stride, coefK, coefV, st);
+}
+
 template <typename TQ>
 int dispatch_attn(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const float *coefK,
                   const float *coefV, const int32_t *t_len, int batch, float scale, void *out,
@@ -737,6 +791,7 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     if (cfg->decode_mode < FAEDKV_DECODE_AUTO || cfg->decode_mode > FAEDKV_DECODE_FFT) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->decode_mode == FAEDKV_DECODE_UMMA && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->decode_mode == FAEDKV_DECODE_FFT && !fft::supported(cfg->n_dft)) return FAEDKV_ERR_UNSUPPORTED;
+    if (cfg->n_sink < 0 || cfg->n_recent < 0 || cfg->n_sink + cfg->n_recent > 1024) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->head_dim != kHeadDim) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FAEDKV_ERR_UNSUPPORTED;
     const int gq = cfg->n_q_heads / cfg->n_kv_heads;
@@ -899,31 +954,7 @@ int faedkv_compress_prefill(faedkv_ctx *ctx, int layer, const void *K, const voi
     if (int r = check_ptrs(ctx, {K, V, coefK, coefV})) return r;
     if (int r = check_tlen(ctx, t_len)) return r;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const faedkv_config &c = ctx->cfg;
-    int mode = c.prefill_mode;
-    if (mode == FAEDKV_PREFILL_AUTO)
-        mode = (c.kv_dtype == FAEDKV_BF16 && umma_prefill_available()) ? FAEDKV_PREFILL_UMMA : FAEDKV_PREFILL_SIMT;
-    int r;
-    if (ctx->prefill_fft) {
-        const int units = batch * c.n_kv_heads;
-        if (c.kv_dtype == FAEDKV_BF16) {
-            r = launch_prefill_fft_tensor<__nv_bfloat16>(ctx, *p, K, units, T, coefK, st);
-            if (r == 0) r = launch_prefill_fft_tensor<__nv_bfloat16>(ctx, *p, V, units, T, coefV, st);
-        } else {
-            r = launch_prefill_fft_tensor<float>(ctx, *p, K, units, T, coefK, st);
-            if (r == 0) r = launch_prefill_fft_tensor<float>(ctx, *p, V, units, T, coefV, st);
-        }
-    } else if (mode == FAEDKV_PREFILL_UMMA) {
-        char msg[256] = {0};
-        r = umma_prefill_launch(ctx->umma, K, V, batch, c.n_kv_heads, T, p->d_bins, p->M, c.n_dft,
-                                c.twiddle_terms == 2 ? 2 : 1, coefK, coefV, ctx->dev_status, st, msg, sizeof(msg));
-        if (r != 0) return fail(ctx, r, "%s", msg);
-    } else if (c.kv_dtype == FAEDKV_BF16) {
-        r = launch_prefill_simt<__nv_bfloat16>(ctx, *p, K, V, batch, T, coefK, coefV, st);
-    } else {
-        r = launch_prefill_simt<float>(ctx, *p, K, V, batch, T, coefK, coefV, st);
-    }
-    if (r) return r;
+    if (int r = prefill_core(ctx, *p, K, V, batch, T, T, coefK, coefV, st)) return r;
     k_set_tlen<<<(batch + 127) / 128, 128, 0, st>>>(t_len, batch, T);
     return launch_check(ctx, "k_set_tlen");
 }
@@ -1013,6 +1044,74 @@ int faedkv_append_decode_attn(faedkv_ctx *ctx, int layer, const void *k_new, con
     if (ctx->cfg.kv_dtype == FAEDKV_BF16)
         return dispatch_attn_fft<__nv_bfloat16, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
     return dispatch_attn_fft<float, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st);
+}
+
+size_t faedkv_window_bytes(const faedkv_ctx *ctx, int batch) {
+    if (ctx == nullptr || batch < 1) return 0;
+    const size_t elem = ctx->cfg.kv_dtype == FAEDKV_BF16 ? 2 : 4;
+    return (size_t)batch * ctx->cfg.n_kv_heads * (ctx->cfg.n_sink + ctx->cfg.n_recent) * kHeadDim * elem;
+}
+
+int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch, int T, float *coefK,
+                            float *coefV, void *winK, void *winV, int32_t *t_len, void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    const faedkv_config &c = ctx->cfg;
+    const int S = c.n_sink, R = c.n_recent;
+    if (K == nullptr || V == nullptr || coefK == nullptr || coefV == nullptr || t_len == nullptr ||
+        (S + R > 0 && (winK == nullptr || winV == nullptr)))
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_prefill_windowed");
+    if (T < S + R || T < 1)
+        return fail(ctx, FAEDKV_ERR_SHAPE, "T = %d must cover the sink and recent windows (%d + %d)", T, S, R);
+    if (int r = check_ptrs(ctx, {K, V, coefK, coefV, winK, winV})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t elem = c.kv_dtype == FAEDKV_BF16 ? 2 : 4;
+    const int mid = T - S - R;
+    if (mid > 0) {
+        // rows [S, T - R) of every unit, at positions 0 .. mid - 1 of the transformed segment (Eq. 10)
+        const char *Km = static_cast<const char *>(K) + (size_t)S * kHeadDim * elem;
+        const char *Vm = static_cast<const char *>(V) + (size_t)S * kHeadDim * elem;
+        if (int r = prefill_core(ctx, *p, Km, Vm, batch, mid, T, coefK, coefV, st)) return r;
+    } else {
+        const size_t bytes = faedkv_coef_bytes(ctx, layer, batch);
+        CUDA_TRY(ctx, cudaMemsetAsync(coefK, 0, bytes, st));
+        CUDA_TRY(ctx, cudaMemsetAsync(coefV, 0, bytes, st));
+    }
+    if (S + R > 0) {
+        dim3 grid(S + R, batch * c.n_kv_heads);
+        if (c.kv_dtype == FAEDKV_BF16)
+            k_window_fill<__nv_bfloat16><<<grid, kHeadDim, 0, st>>>(static_cast<const __nv_bfloat16 *>(K), static_cast<const __nv_bfloat16 *>(V),
+                                                                   static_cast<__nv_bfloat16 *>(winK), static_cast<__nv_bfloat16 *>(winV), T, S, R);
+        else
+            k_window_fill<float><<<grid, kHeadDim, 0, st>>>(static_cast<const float *>(K), static_cast<const float *>(V),
+                                                           static_cast<float *>(winK), static_cast<float *>(winV), T, S, R);
+        if (int r = launch_check(ctx, "k_window_fill")) return r;
+    }
+    k_set_tlen<<<(batch + 127) / 128, 128, 0, st>>>(t_len, batch, T);
+    return launch_check(ctx, "k_set_tlen");
+}
+
+int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new, const void *q, int batch,
+                         float *coefK, float *coefV, void *winK, void *winV, int32_t *t_len, float scale, void *out,
+                         void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    if (k_new == nullptr || v_new == nullptr || q == nullptr || coefK == nullptr || coefV == nullptr ||
+        winK == nullptr || winV == nullptr || t_len == nullptr || out == nullptr)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_step_windowed");
+    if (!(scale >= 0.0f)) return fail(ctx, FAEDKV_ERR_INVALID_ARG, "scale must be >= 0");
+    if (int r = check_ptrs(ctx, {k_new, v_new, q, coefK, coefV, winK, winV, out})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    if (!ctx->use_fft)
+        return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "the windowed step needs the FFT-shaped decode path (P a power of two in [64, 2^19])");
+    if (scale == 0.0f) scale = 1.0f / sqrtf((float)ctx->cfg.head_dim);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (ctx->cfg.kv_dtype == FAEDKV_BF16)
+        return dispatch_attn_fft<__nv_bfloat16, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+    return dispatch_attn_fft<float, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
 }
 
 unsigned long long faedkv_launch_count(const faedkv_ctx *ctx) { return ctx ? ctx->launches : 0ULL; }

@@ -17,6 +17,7 @@
 #include "common.cuh"
 #include "k_attn.cuh"
 #include "k_fft.cuh"
+#include "k_window.cuh"
 
 namespace faedkv {
 
@@ -26,7 +27,7 @@ template <typename TQ, int GQ, bool APPEND>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restrict__ k_new,
           const int32_t *__restrict__ t_len, const int32_t *__restrict__ bins, float2 *__restrict__ Qs,
-          int M, int H, int HQ, int Gp, uint32_t P, float scale_over_P) {
+          int M, int H, int HQ, int Gp, uint32_t P, float scale_over_P, FoldSrc fold) {
     constexpr int KB = 16 / GQ;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
@@ -46,9 +47,12 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
             if (k0 + kk < M) row[kk][pl] = ld_stream(base + pl * plane + (size_t)(k0 + kk) * kHeadDim + lane * 4);
         }
     if (APPEND) {
-        // C_K[k, c] += k_new[c] * e^{-j w k t}: same arithmetic as k_append
-        const uint32_t t = (uint32_t)t_len[b] % P;
-        const float4 x = load4(k_new + (size_t)bh * kHeadDim + lane * 4);
+        // C_K[k, c] += x[c] * e^{-j w k t}: same arithmetic as k_append; x is the call's new token, or with a
+        // recent window the token that leaves it (k_new then points at the window tensor)
+        size_t xrow;
+        uint32_t t;
+        fold_locate(fold, t_len[b], bh, P, xrow, t);
+        const float4 x = load4(k_new + xrow * kHeadDim + lane * 4);
 #pragma unroll
         for (int kk = 0; kk < KB; ++kk) {
             if (k0 + kk >= M) continue;
@@ -233,7 +237,8 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
 template <int LG>
 __global__ void __launch_bounds__(fft::kThreads)
 k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restrict__ mloc,
-             const float *__restrict__ sloc, int lgMT, float2 *__restrict__ Zf, float *__restrict__ colsum, int lgKT) {
+             const float *__restrict__ sloc, int lgMT, float2 *__restrict__ Zf, float *__restrict__ colsum, int lgKT,
+             int n_extra) {
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N1
     extern __shared__ float2 fft_smem[];
@@ -246,11 +251,14 @@ k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restr
     float *fac = reinterpret_cast<float *>(tw + NF);  // [n_tiles][16]
     const int k1_0 = blockIdx.x << lgKT, g0 = blockIdx.y * kCW;
     const int n_tiles = NF >> lgMT;
+    // n_extra = 1: row n_tiles of mloc / sloc holds the statistics of the sink + recent window, which joins
+    // the softmax as one more tile; its factor is handed to the output kernel in colsum[Gp + col]
+    const int n_stat = n_tiles + n_extra;
     fill_twiddles(tw, NF);
     const int c = threadIdx.x & (kCW - 1);
     {
         float mx = -INFINITY;
-        for (int ti = threadIdx.x >> kLgCW; ti < n_tiles; ti += kThreads / kCW) mx = fmaxf(mx, mloc[(size_t)ti * g.Gp + g0 + c]);
+        for (int ti = threadIdx.x >> kLgCW; ti < n_stat; ti += kThreads / kCW) mx = fmaxf(mx, mloc[(size_t)ti * g.Gp + g0 + c]);
         red[threadIdx.x] = mx;
         __syncthreads();
         if (threadIdx.x < kCW) {
@@ -262,11 +270,14 @@ k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restr
         __syncthreads();
         const float m = mg[c];
         float part = 0.f;
-        for (int ti = threadIdx.x >> kLgCW; ti < n_tiles; ti += kThreads / kCW) {
+        for (int ti = threadIdx.x >> kLgCW; ti < n_stat; ti += kThreads / kCW) {
             const float ml = mloc[(size_t)ti * g.Gp + g0 + c];
             const float f = ml == -INFINITY ? 0.f : __expf(ml - m);
             fac[ti * kCW + c] = f;
-            if (blockIdx.x == 0) part += f * sloc[(size_t)ti * g.Gp + g0 + c];
+            if (blockIdx.x == 0) {
+                part += f * sloc[(size_t)ti * g.Gp + g0 + c];
+                if (ti == n_tiles) colsum[g.Gp + g0 + c] = f;
+            }
         }
         if (blockIdx.x == 0) {
             __syncthreads();
@@ -305,7 +316,7 @@ inline size_t afft_smem_mid(int lg, int lgMT) {
 }
 inline size_t afft_smem_fwd_b(int lg, int lgKT, int lgMT) {
     const size_t nf = (size_t)1 << lg, tile = nf << (lgKT + fft::kLgCW);
-    return (fft::exchange_buffers(lg) * tile + nf) * sizeof(float2) + ((nf >> lgMT) * fft::kCW) * sizeof(float);
+    return (fft::exchange_buffers(lg) * tile + nf) * sizeof(float2) + (((nf >> lgMT) + 1) * fft::kCW) * sizeof(float);
 }
 
 // ---- (5) ------------------------------------------------------------------------------------------
@@ -322,7 +333,8 @@ __global__ void __launch_bounds__(kAttnWarps * 32)
 k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t *__restrict__ t_len,
                const float2 *__restrict__ Zf, const float *__restrict__ colsum, const int32_t *__restrict__ bins,
                float *__restrict__ partial, unsigned int *__restrict__ tickets, TQ *__restrict__ out,
-               int M, int H, int HQ, fft::Geometry g, int bins_per_slice, float inv_P) {
+               int M, int H, int HQ, fft::Geometry g, int bins_per_slice, float inv_P, FoldSrc fold,
+               const float *__restrict__ o_win, int bump) {
     using namespace fft;
     // the weights of a chunk and the final cross-warp reduction share one buffer
     constexpr size_t kWgtBytes = (size_t)kOutChunk * GQ * sizeof(float2) + (APPEND ? kOutChunk * sizeof(float2) : 0);
@@ -342,8 +354,9 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
     float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
     uint32_t t = 0;
     if (APPEND) {
-        x = load4(v_new + (size_t)bh * kHeadDim + lane * 4);
-        t = (uint32_t)t_len[b] % g.P;
+        size_t xrow;
+        fold_locate(fold, t_len[b], bh, g.P, xrow, t);
+        x = load4(v_new + xrow * kHeadDim + lane * 4);
     }
     float4 acc[GQ];
 #pragma unroll
@@ -436,9 +449,12 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
             float s = 0.f;
             for (int sl = 0; sl < (int)gridDim.x; ++sl)
                 s += __ldcg(partial + (((size_t)bh * gridDim.x + sl) * GQ + q) * kHeadDim + c);
-            store1(out + (size_t)(gcol + q) * kHeadDim + c, s * inv_P / colsum[gcol + q]);
+            s *= inv_P;
+            // the sink + recent window's share of the same softmax (its factor sits behind the normalisers)
+            if (o_win != nullptr) s = fmaf(o_win[(size_t)(gcol + q) * kHeadDim + c], colsum[g.Gp + gcol + q], s);
+            store1(out + (size_t)(gcol + q) * kHeadDim + c, s / colsum[gcol + q]);
         }
-        if (APPEND) {
+        if (APPEND && bump) {
             // every CTA of this sequence has read t_len before taking its ticket; the last CTA of the
             // sequence's last kv head advances the counter once all H heads are through
             if (threadIdx.x == 0) {

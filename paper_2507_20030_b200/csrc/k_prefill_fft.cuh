@@ -17,10 +17,10 @@
 
 namespace faedkv {
 
-// grid = (N1 / MT, cols / 16); block = 256.  x: [units][T][128] of the tensor.
+// grid = (N1 / MT, cols / 16); block = 256.  x: rows of the tensor, T rows per unit, units T_stride rows apart.
 template <int LG, typename TIn>
 __global__ void __launch_bounds__(fft::kThreads)
-k_pfft_fwd_a(fft::Geometry g, const TIn *__restrict__ x, int T, int unit0, float2 *__restrict__ U, int lgMT) {
+k_pfft_fwd_a(fft::Geometry g, const TIn *__restrict__ x, int T, int T_stride, int unit0, float2 *__restrict__ U, int lgMT) {
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N2
     extern __shared__ float2 fft_smem[];
@@ -37,7 +37,7 @@ k_pfft_fwd_a(fft::Geometry g, const TIn *__restrict__ x, int T, int unit0, float
         tab_i[e] = unit_phasor((uint32_t)((m1_0 + mt) * r), (uint32_t)g.N);
     }
     __syncthreads();
-    const TIn *xu = x + (size_t)(unit0 + (g0 >> 7)) * T * kHeadDim + (g0 & (kHeadDim - 1));
+    const TIn *xu = x + (size_t)(unit0 + (g0 >> 7)) * T_stride * kHeadDim + (g0 & (kHeadDim - 1));
     const bool wraps = T > (int)g.P;                                     // uniform: positions beyond P fold back
     auto load = [&](int m2, int cidx) {
         const int c = cidx & (kCW - 1);

@@ -304,10 +304,13 @@ inline int umma_resolve_encode(UmmaPrefillState &st, char *msg, size_t n) {
     return 0;
 }
 
-inline int umma_make_map(UmmaPrefillState &st, CUtensorMap *map, const void *base, int units, int T, char *msg, size_t n) {
+// T rows of each unit are transformed; consecutive units are T_stride rows apart (T_stride >= T: the
+// transformed rows may be a window of a longer tensor).
+inline int umma_make_map(UmmaPrefillState &st, CUtensorMap *map, const void *base, int units, int T, int T_stride, char *msg,
+                         size_t n) {
     if (int r = umma_resolve_encode(st, msg, n)) return r;
     cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)T, (cuuint64_t)units};
-    cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)T * kHeadDim * 2};
+    cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)T_stride * kHeadDim * 2};
     cuuint32_t box[3] = {64, (cuuint32_t)prefill::kTileTok, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = st.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
@@ -343,13 +346,13 @@ inline int umma_launch_t(UmmaPrefillState &st, const CUtensorMap &mK, const CUte
     return 0;
 }
 
-inline int umma_prefill_launch(UmmaPrefillState &st, const void *K, const void *V, int batch, int H, int T,
+inline int umma_prefill_launch(UmmaPrefillState &st, const void *K, const void *V, int batch, int H, int T, int T_stride,
                                const int32_t *d_bins, int M, int P, int terms, float *coefK, float *coefV,
                                unsigned int *status, cudaStream_t stream, char *msg, size_t n) {
     CUtensorMap mK, mV;
     const int units = batch * H;
-    if (int r = umma_make_map(st, &mK, K, units, T, msg, n)) return r;
-    if (int r = umma_make_map(st, &mV, V, units, T, msg, n)) return r;
+    if (int r = umma_make_map(st, &mK, K, units, T, T_stride, msg, n)) return r;
+    if (int r = umma_make_map(st, &mV, V, units, T, T_stride, msg, n)) return r;
     if (terms == 2) return umma_launch_t<2>(st, mK, mV, units, T, d_bins, M, P, coefK, coefV, status, stream, msg, n);
     return umma_launch_t<1>(st, mK, mV, units, T, d_bins, M, P, coefK, coefV, status, stream, msg, n);
 }

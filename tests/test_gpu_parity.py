@@ -517,3 +517,78 @@ def test_prefill_fft_matches_oracle(fk, oracle, dtype, P, T, M, B, H):
     errV = rel_l2(to_np64(cV), oracle_compress(oracle, V, P, bins))
     assert errK <= REL_L2_F32 and errV <= REL_L2_F32, (errK, errV)
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- sink + recent window
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,T,M,B,H,HQ,S,R,steps", [
+    (256, 200, 40, 2, 2, 8, 10, 50, 12),      # the paper's S = 10, R = 50; GQA 4
+    (128, 64, 65, 1, 3, 3, 4, 7, 20),         # every bin retained; MHA; the ring turns over more than twice
+    (512, 520, 33, 2, 1, 2, 0, 16, 5),        # no sink; the transformed segment is longer than P (wraps)
+    (64, 30, 9, 1, 2, 4, 6, 0, 6),            # no ring: the new token itself is folded
+    (1024, 60, 24, 2, 2, 4, 10, 50, 4),       # T = S + R: the transformed segment starts empty
+])
+def test_windowed_step_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, S, R, steps):
+    """Prefill with sink + recent window, then decode steps: attention outputs, planes, window contents
+    and counters against the oracle's WindowedUnit, unit by unit."""
+    from paper_2507_20030_b200 import synth
+    GQ = HQ // H
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                     prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R)
+    mask = _random_mask(P, M, 13 * P + T)
+    mask[0] = 1
+    M = int(mask.sum())
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    assert ctx._lib.faedkv_window_bytes(ctx._h, B) == B * H * (S + R) * 128 * (4 if dtype == torch.float32 else 2)
+    K, V = _make(51 + P + T, B, H, T, dtype)
+    V = (V * 0.25).to(dtype)                  # keeps bf16 outputs on a grid finer than the absolute tolerance
+    units = {(b, h): oracle.WindowedUnit(P, bins, S, R) for b in range(B) for h in range(H)}
+    for (b, h), u in units.items():
+        u.prefill(to_np64(K[b, h]), to_np64(V[b, h]))
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    cK.fill_(float("nan")); cV.fill_(float("nan"))
+    wK, wV = ctx.alloc_window(B), ctx.alloc_window(B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.prefill_windowed(0, K.cuda(), V.cuda(), cK, cV, wK, wV, t_len)
+    out = torch.empty((B, HQ, 128), dtype=dtype, device="cuda")
+    for s in range(steps):
+        k, v = synth.make_token(77, s, B, H, 128, pos=T + s, dtype=dtype)
+        v = (v * 0.25).to(dtype)
+        q = synth.make_q(77, s, B, HQ, 128, dtype=dtype)
+        ctx.step_windowed(0, k.cuda(), v.cuda(), q.cuda(), cK, cV, wK, wV, t_len, out)
+        torch.cuda.synchronize()
+        got = to_np64(out)
+        for (b, h), u in units.items():
+            u.step(to_np64(k[b, h]), to_np64(v[b, h]))
+            want = u.attention(to_np64(q[b, h * GQ:(h + 1) * GQ]))
+            err = np.abs(got[b, h * GQ:(h + 1) * GQ] - want).max()
+            assert err <= ATTN_MAX_ABS, (s, b, h, err)
+    assert t_len.tolist() == [T + steps] * B and ctx.device_status() == 0
+    gK, gV, gwK = to_np64(cK), to_np64(cV), to_np64(wK)
+    for (b, h), u in units.items():
+        assert rel_l2(gK[b, h], np.stack(u.CK)) <= REL_L2_F32 and rel_l2(gV[b, h], np.stack(u.CV)) <= REL_L2_F32
+        assert np.array_equal(gwK[b, h, :S], u.sinkK)
+        if R > 0:                             # ring slot of token n is (n - S) mod R
+            t = T + steps
+            for j, n in enumerate(range(t - R, t)):
+                assert np.array_equal(gwK[b, h, S + (n - S) % R], u.recentK[j]), (b, h, n)
+    ctx.close()
+
+
+def test_windowed_rejects_short_prefill_and_non_fft_grids(fk):
+    ctx = fk.Context(n_layers=1, n_kv_heads=1, n_q_heads=1, n_dft=100, max_batch=1, kv_dtype=fk.F32, n_sink=4, n_recent=8)
+    ctx.plan(0, _mask_from_bins(100, [0, 1, 2]))
+    K = torch.zeros(1, 1, 11, 128, device="cuda")
+    cK, w = ctx.alloc_coef(0, 1), ctx.alloc_window(1)
+    t = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx.prefill_windowed(0, K, K, cK, cK, w, w, t)
+    assert e.value.code == -3                                   # T < S + R
+    K = torch.zeros(1, 1, 20, 128, device="cuda")
+    ctx.prefill_windowed(0, K, K, cK, cK, w, w, t)
+    x = torch.zeros(1, 1, 128, device="cuda")
+    with pytest.raises(fk.FaedkvError) as e:
+        ctx.step_windowed(0, x, x, x, cK, cK, w, w, t, x.clone())
+    assert e.value.code == -4                                   # P = 100 has no FFT-shaped path
+    ctx.close()

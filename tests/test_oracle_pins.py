@@ -396,3 +396,70 @@ def test_mixed_mask_independent_restatement(oracle):
     want = sorted(list(range(n_low)) + [c * g + b for c in chosen for b in range(g)])
     got = oracle.plan(P, oracle.mask_mixed(P, M, layer, seed))
     np.testing.assert_array_equal(got, want)
+
+
+# ----------------------------------------------------------------------------- sink + recent window
+def _numpy_attention(q, K, V, scale):
+    s = (q @ K.T) * scale
+    s -= s.max(axis=1, keepdims=True)
+    p = np.exp(s)
+    return (p / p.sum(axis=1, keepdims=True)) @ V
+
+
+@pytest.mark.parametrize("S,R", [(3, 5), (0, 4), (6, 0), (0, 0)])
+def test_windowed_all_bins_is_full_attention(oracle, S, R):
+    """Every bin retained and the sequence shorter than the grid: sink + exact reconstruction + recent is
+    the whole cache, so the windowed workflow equals textbook attention over all tokens (numpy),
+    whatever S and R, before and after decode steps."""
+    P, T, d, G, steps = 64, 30, 8, 3, 9
+    rng = np.random.default_rng(S * 10 + R)
+    K, V = rng.standard_normal((T + steps, d)), rng.standard_normal((T + steps, d))
+    bins = oracle.plan(P, np.ones(P // 2 + 1, dtype=np.uint8))
+    u = oracle.WindowedUnit(P, bins, S, R)
+    u.prefill(K[:T], V[:T])
+    for s in range(steps + 1):
+        q = rng.standard_normal((G, d))
+        got = u.attention(q, 0.3)
+        want = _numpy_attention(q, K[:T + s], V[:T + s], 0.3)
+        assert np.abs(got - want).max() < 1e-11, (s, np.abs(got - want).max())
+        if s < steps:
+            u.step(K[T + s], V[T + s])
+    assert u.t == T + steps
+
+
+def test_windowed_without_window_is_plain_decode(oracle):
+    """S = R = 0: prefill, step and attention reduce to compress, append and decode_attn."""
+    P, T, d, G = 48, 40, 6, 2
+    rng = np.random.default_rng(5)
+    K, V = rng.standard_normal((T + 1, d)), rng.standard_normal((T + 1, d))
+    mask = np.zeros(P // 2 + 1, dtype=np.uint8)
+    mask[[0, 1, 2, 5, 9, 24]] = 1
+    bins = oracle.plan(P, mask)
+    u = oracle.WindowedUnit(P, bins, 0, 0)
+    u.prefill(K[:T], V[:T])
+    u.step(K[T], V[T])
+    re, im = oracle.compress(K[:T + 1], P, bins)
+    assert np.abs(u.CK[0] - re).max() < 1e-11 and np.abs(u.CK[1] - im).max() < 1e-11
+    q = rng.standard_normal((G, d))
+    vre, vim = oracle.compress(V[:T + 1], P, bins)
+    want = oracle.decode_attn(q, re, im, vre, vim, P, bins, T + 1, 0.25)
+    assert np.abs(u.attention(q, 0.25) - want).max() < 1e-12
+
+
+def test_windowed_folds_the_token_that_leaves_the_window(oracle):
+    """After steps the transformed segment is exactly the DFT of tokens [S, t - R) at positions n - S
+    (Eq. 10 and Eq. 12 agree), and the window holds the last R tokens in order."""
+    P, T, d, S, R, steps = 32, 20, 4, 2, 3, 7
+    rng = np.random.default_rng(11)
+    K, V = rng.standard_normal((T + steps, d)), rng.standard_normal((T + steps, d))
+    mask = np.zeros(P // 2 + 1, dtype=np.uint8)
+    mask[[0, 3, 4, 16]] = 1
+    bins = oracle.plan(P, mask)
+    u = oracle.WindowedUnit(P, bins, S, R)
+    u.prefill(K[:T], V[:T])
+    for s in range(steps):
+        u.step(K[T + s], V[T + s])
+    t = T + steps
+    re, im = oracle.compress(K[S:t - R], P, bins)
+    assert np.abs(u.CK[0] - re).max() < 1e-11 and np.abs(u.CK[1] - im).max() < 1e-11
+    assert np.array_equal(np.stack(u.recentV), V[t - R:t]) and np.array_equal(u.sinkK, K[:S])
