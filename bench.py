@@ -189,7 +189,8 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     as one CUDA graph (launch gaps excluded) and, for the fused call, also launched eagerly."""
     NL, H, HQ, B, T, M = (W[k] for k in ("n_layers", "n_kv_heads", "n_q_heads", "batch", "T", "M"))
     P, D = T, 128
-    ctx = binding.Context(n_layers=NL, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=binding.BF16)
+    ctx = binding.Context(n_layers=NL, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=binding.BF16,
+                          n_sink=10, n_recent=50)       # the paper's window sizes; only step_windowed looks at them
     seed = synth.config_seed(W["config"])
     cKs, cVs, tls = [], [], []
     for l in range(NL):
@@ -204,14 +205,18 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     k_new, v_new = synth.make_token(seed, 0, B, H, D, pos=T, dtype=torch.bfloat16, device=dev)
     q = synth.make_q(seed, 0, B, HQ, D, dtype=torch.bfloat16, device=dev)
     out = torch.empty((B, HQ, D), dtype=torch.bfloat16, device=dev)
+    # windows of the paper's workflow (sink 10 + recent 50), filled with tokens of the same distributions
+    wK, wV = synth.make_kv(seed + 7, B, H, 60, D, pos0=T - 60, dtype=torch.bfloat16, device=dev)
     loops = {
+        "step_windowed": lambda: [ctx.step_windowed(l, k_new, v_new, q, cKs[l], cVs[l], wK, wV, tls[l], out) for l in range(NL)],
         "append": lambda: [ctx.append(l, k_new, v_new, cKs[l], cVs[l], tls[l]) for l in range(NL)],
         "decode_attn": lambda: [ctx.decode_attn(l, q, cKs[l], cVs[l], tls[l], out) for l in range(NL)],
         "append_decode_attn": lambda: [ctx.append_decode_attn(l, k_new, v_new, q, cKs[l], cVs[l], tls[l], out)
                                        for l in range(NL)],
     }
     coef_bytes = 2 * B * H * 2 * M * D * 4                      # K and V planes of one layer
-    alg_bytes = {"append": 2 * coef_bytes, "decode_attn": coef_bytes, "append_decode_attn": 2 * coef_bytes}
+    alg_bytes = {"append": 2 * coef_bytes, "decode_attn": coef_bytes, "append_decode_attn": 2 * coef_bytes,
+                 "step_windowed": 2 * coef_bytes}
     res = {"workload": W["name"], "iters": iters, "planes_bytes_per_layer": coef_bytes,
            "l2": "32 layers cycled: %.0f MiB of planes per layer" % (coef_bytes / 2 ** 20)}
     side = torch.cuda.Stream()
