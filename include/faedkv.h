@@ -220,6 +220,40 @@ int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const vo
                          const void *q, int batch, float *coefK, float *coefV, void *winK,
                          void *winV, int32_t *t_len, float scale, void *out, void *stream);
 
+/* ---- frequency ablation and bin selection (Sec. 3.2) -----------------------------------------------
+ * The paper chooses each layer's retained bins once per model: the P two-sided bins are cut into C
+ * contiguous chunks (C = 22 in the paper), each chunk is zeroed in turn in the DFT of the layer's K and
+ * V caches (Eq. 6), the perplexity change Delta is measured, and the r*C chunks with the largest Delta
+ * are kept.  The perplexity runs need a model and a corpus and are the caller's; these calls are the
+ * rest of the procedure. */
+
+/* Two-sided bins [*lo, *hi) of chunk `chunk` of n_chunks: chunks of floor(P / n_chunks) bins, the
+ * last one running to P.  host: lo, hi. */
+int faedkv_chunk_range(int n_dft, int n_chunks, int chunk, int *lo, int *hi);
+
+/* One-sided view of zeroing the two-sided bins [lo, hi) of a real signal.  mask_out, gain_out: host,
+ * length P/2 + 1.  mask_out[k] = 1 when bin k or its mirror P - k is zeroed; gain_out[k] = the share
+ * of that conjugate pair's real component that disappears from Re(IDFT): 1 when both are zeroed (or k
+ * is its own mirror), 1/2 when only one of them is, 0 elsewhere. */
+int faedkv_ablation_bins(int n_dft, int lo, int hi, uint8_t *mask_out, float *gain_out);
+
+/* Greedy selection: keeps the n_keep = max(1, floor(ratio * n_chunks + 1/2)) chunks with the largest
+ * delta (host, n_chunks doubles; ties go to the lower chunk index) and writes the one-sided keep-mask
+ * for faedkv_plan (a bin is kept when it or its mirror lies in a kept chunk).  *n_keep_out may be NULL. */
+int faedkv_mask_from_scores(int n_dft, int n_chunks, const double *delta, double ratio,
+                            uint8_t *mask_out, int *n_keep_out);
+
+/* The ablated caches (Eq. 6, then Eq. 5, real part):  X_out = X - sum_i gain[i] * (component of
+ * retained bin i of X), for X = K and X = V, [batch][n_kv_heads][T][head_dim], T <= P (rows beyond T
+ * count as zero; the paper's N is the sequence length, i.e. create the context with n_dft = T).
+ * The layer must be planned with the mask from faedkv_ablation_bins; gain: DEVICE float[M], the
+ * gains of the retained bins in ascending bin order.  wsK, wsV (faedkv_coef_bytes each) and ws_len
+ * (int32[batch]) are workspaces the call overwrites.  Runs compress_prefill, a scaling of the planes,
+ * reconstruct and a subtraction on `stream`. */
+int faedkv_ablate(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch, int T,
+                  const float *gain, float *wsK, float *wsV, int32_t *ws_len, void *K_out, void *V_out,
+                  void *stream);
+
 /* Device-side status word of the context (host read; synchronises `stream`):
  * 0, or a nonzero code left by a kernel whose bounded wait on an mbarrier gave
  * up.  Such a kernel returns early instead of hanging; its output is invalid. */

@@ -283,3 +283,57 @@ class WindowedUnit:
         Kt = np.concatenate([p for p in parts_k if p.shape[0] > 0], axis=0)
         Vt = np.concatenate([p for p in parts_v if p.shape[0] > 0], axis=0)
         return attention_dense(q, Kt, Vt, scale)
+
+
+# ---------------------------------------------------------------------------------------------------
+# Frequency ablation and bin selection (Sec. 3.2).  Integer logic in plain Python; the ablation itself is
+# the definition written out with numpy's float64 FFT as the library step.
+def chunk_range(P: int, C: int, c: int) -> tuple[int, int]:
+    """Two-sided bins [lo, hi) of chunk c when the P bins are cut into C contiguous chunks of P // C bins;
+    the last chunk takes the remainder."""
+    assert 1 <= C <= P and 0 <= c < C
+    w = P // C
+    return c * w, (P if c == C - 1 else (c + 1) * w)
+
+
+def ablate(x: np.ndarray, P: int, lo: int, hi: int) -> np.ndarray:
+    """Eq. 6 then Eq. 5: DFT of x [T, d] (T <= P, zero-padded to the grid) along the token axis, bins
+    lo <= k < hi set to zero, inverse DFT, real part, first T rows."""
+    x = _f64arr(x)
+    T = x.shape[0]
+    assert T <= P
+    X = np.fft.fft(x, n=P, axis=0)
+    X[lo:hi] = 0.0
+    return np.fft.ifft(X, axis=0).real[:T]
+
+
+def ablation_bins(P: int, lo: int, hi: int) -> tuple[np.ndarray, np.ndarray]:
+    """One-sided view of zeroing two-sided bins [lo, hi) of a REAL signal: mask[k] = 1 for every
+    k in [0, P/2] whose bin k or mirror P-k is zeroed, gain[k] = the share of that bin's real component
+    that disappears: 1 when both k and P-k are zeroed (or k is its own mirror), else 1/2."""
+    n1 = P // 2 + 1
+    mask = np.zeros(n1, dtype=np.uint8)
+    gain = np.zeros(n1, dtype=np.float32)
+    for k in range(n1):
+        a = lo <= k < hi
+        b = lo <= (P - k) % P < hi
+        if a or b:
+            mask[k] = 1
+            gain[k] = 1.0 if (a and b) else 0.5
+    return mask, gain
+
+
+def mask_from_scores(P: int, C: int, delta, ratio: float) -> tuple[np.ndarray, int]:
+    """Greedy selection: keep the n_keep = max(1, floor(ratio * C + 1/2)) chunks with the largest
+    perplexity change delta (ties: the lower chunk index wins); a one-sided bin is kept when it or its
+    mirror lies in a kept chunk."""
+    delta = [float(v) for v in delta]
+    assert len(delta) == C
+    n_keep = max(1, int(np.floor(ratio * C + 0.5)))
+    n_keep = min(n_keep, C)
+    order = sorted(range(C), key=lambda c: (-delta[c], c))
+    keep2 = np.zeros(P, dtype=np.uint8)
+    for c in order[:n_keep]:
+        lo, hi = chunk_range(P, C, c)
+        keep2[lo:hi] = 1
+    return fold_two_sided(P, keep2), n_keep

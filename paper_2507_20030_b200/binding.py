@@ -27,7 +27,8 @@ EXPORTS = [
     "faedkv_create", "faedkv_destroy", "faedkv_last_error", "faedkv_plan", "faedkv_n_bins",
     "faedkv_get_bins", "faedkv_coef_bytes", "faedkv_mask_lowpass", "faedkv_mask_mixed",
     "faedkv_compress_prefill", "faedkv_append", "faedkv_reconstruct", "faedkv_decode_attn",
-    "faedkv_append_decode_attn", "faedkv_window_bytes", "faedkv_prefill_windowed", "faedkv_step_windowed",
+    "faedkv_append_decode_attn", "faedkv_chunk_range", "faedkv_ablation_bins", "faedkv_mask_from_scores", "faedkv_ablate",
+    "faedkv_window_bytes", "faedkv_prefill_windowed", "faedkv_step_windowed",
     "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
 ]
 
@@ -89,6 +90,14 @@ def load() -> ctypes.CDLL:
     lib.faedkv_decode_attn.restype = _int
     lib.faedkv_append_decode_attn.argtypes = [_vp, _int, _vp, _vp, _vp, _int, _vp, _vp, _vp, ctypes.c_float, _vp, _vp]
     lib.faedkv_append_decode_attn.restype = _int
+    lib.faedkv_chunk_range.argtypes = [_int, _int, _int, ctypes.POINTER(_int), ctypes.POINTER(_int)]
+    lib.faedkv_chunk_range.restype = _int
+    lib.faedkv_ablation_bins.argtypes = [_int, _int, _int, _vp, _vp]
+    lib.faedkv_ablation_bins.restype = _int
+    lib.faedkv_mask_from_scores.argtypes = [_int, _int, _vp, ctypes.c_double, _vp, ctypes.POINTER(_int)]
+    lib.faedkv_mask_from_scores.restype = _int
+    lib.faedkv_ablate.argtypes = [_vp, _int, _vp, _vp, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+    lib.faedkv_ablate.restype = _int
     lib.faedkv_window_bytes.argtypes = [_vp, _int]
     lib.faedkv_window_bytes.restype = ctypes.c_size_t
     lib.faedkv_prefill_windowed.argtypes = [_vp, _int, _vp, _vp, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -120,6 +129,35 @@ def mask_mixed(n_dft: int, n_keep: int, layer: int, seed: int) -> np.ndarray:
     if rc != 0:
         raise FaedkvError(rc, "faedkv_mask_mixed rejected its arguments")
     return out
+
+
+def chunk_range(n_dft: int, n_chunks: int, chunk: int) -> tuple[int, int]:
+    lo, hi = _int(0), _int(0)
+    rc = load().faedkv_chunk_range(n_dft, n_chunks, chunk, ctypes.byref(lo), ctypes.byref(hi))
+    if rc != 0:
+        raise FaedkvError(rc, "faedkv_chunk_range rejected its arguments")
+    return lo.value, hi.value
+
+
+def ablation_bins(n_dft: int, lo: int, hi: int) -> tuple[np.ndarray, np.ndarray]:
+    mask = np.zeros(n_dft // 2 + 1, dtype=np.uint8)
+    gain = np.zeros(n_dft // 2 + 1, dtype=np.float32)
+    rc = load().faedkv_ablation_bins(n_dft, lo, hi, mask.ctypes.data, gain.ctypes.data)
+    if rc != 0:
+        raise FaedkvError(rc, "faedkv_ablation_bins rejected its arguments")
+    return mask, gain
+
+
+def mask_from_scores(n_dft: int, n_chunks: int, delta, ratio: float) -> tuple[np.ndarray, int]:
+    d = np.ascontiguousarray(delta, dtype=np.float64)
+    if d.shape != (n_chunks,):
+        raise ValueError("delta must have one entry per chunk")
+    mask = np.zeros(n_dft // 2 + 1, dtype=np.uint8)
+    n_keep = _int(0)
+    rc = load().faedkv_mask_from_scores(n_dft, n_chunks, d.ctypes.data, float(ratio), mask.ctypes.data, ctypes.byref(n_keep))
+    if rc != 0:
+        raise FaedkvError(rc, "faedkv_mask_from_scores rejected its arguments")
+    return mask, n_keep.value
 
 
 def decode_attn_static(n_dft: int, n_kv_heads: int, n_q_heads: int, kv_dtype: int, bins, q, coefK, coefV,
@@ -261,6 +299,12 @@ class Context:
         self._check(self._lib.faedkv_append_decode_attn(
             self._h, layer, _ptr(k_new), _ptr(v_new), _ptr(q), batch, _ptr(coefK), _ptr(coefV), _ptr(t_len),
             float(scale), _ptr(out), _stream(stream)))
+
+    def ablate(self, layer, K, V, gain, wsK, wsV, ws_len, K_out, V_out, stream=None):
+        batch, T = K.shape[0], K.shape[2]
+        self._check(self._lib.faedkv_ablate(
+            self._h, layer, _ptr(K), _ptr(V), batch, T, _ptr(gain), _ptr(wsK), _ptr(wsV), _ptr(ws_len),
+            _ptr(K_out), _ptr(V_out), _stream(stream)))
 
     # -- sink + recent window
     def alloc_window(self, batch: int, device="cuda") -> torch.Tensor:

@@ -1,5 +1,7 @@
 // Host side of the FAEDKV C ABI: context, per-layer plans, argument checks and
 // kernel launches.  See include/faedkv.h for the contract of every call.
+#include <algorithm>
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -18,6 +20,7 @@
 #include "k_attn_fft.cuh"
 #include "k_recon_fft.cuh"
 #include "k_prefill_fft.cuh"
+#include "k_ablate.cuh"
 
 using namespace faedkv;
 
@@ -1112,6 +1115,85 @@ int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const vo
     if (ctx->cfg.kv_dtype == FAEDKV_BF16)
         return dispatch_attn_fft<__nv_bfloat16, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
     return dispatch_attn_fft<float, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+}
+
+int faedkv_chunk_range(int n_dft, int n_chunks, int chunk, int *lo, int *hi) {
+    if (n_dft < 2 || n_chunks < 1 || n_chunks > n_dft || chunk < 0 || chunk >= n_chunks || lo == nullptr || hi == nullptr)
+        return FAEDKV_ERR_INVALID_ARG;
+    const int w = n_dft / n_chunks;
+    *lo = chunk * w;
+    *hi = chunk == n_chunks - 1 ? n_dft : (chunk + 1) * w;
+    return FAEDKV_OK;
+}
+
+int faedkv_ablation_bins(int n_dft, int lo, int hi, uint8_t *mask_out, float *gain_out) {
+    if (n_dft < 2 || lo < 0 || hi > n_dft || lo >= hi || mask_out == nullptr || gain_out == nullptr)
+        return FAEDKV_ERR_INVALID_ARG;
+    for (int k = 0; k <= n_dft / 2; ++k) {
+        const int mirror = (n_dft - k) % n_dft;
+        const bool a = lo <= k && k < hi, b = lo <= mirror && mirror < hi;
+        mask_out[k] = (a || b) ? 1 : 0;
+        gain_out[k] = (a && b) ? 1.0f : ((a || b) ? 0.5f : 0.0f);
+    }
+    return FAEDKV_OK;
+}
+
+int faedkv_mask_from_scores(int n_dft, int n_chunks, const double *delta, double ratio, uint8_t *mask_out,
+                            int *n_keep_out) {
+    if (n_dft < 2 || n_chunks < 1 || n_chunks > n_dft || delta == nullptr || mask_out == nullptr || !(ratio >= 0.0))
+        return FAEDKV_ERR_INVALID_ARG;
+    int n_keep = (int)std::floor(ratio * n_chunks + 0.5);
+    if (n_keep < 1) n_keep = 1;
+    if (n_keep > n_chunks) n_keep = n_chunks;
+    std::vector<int> order(n_chunks);
+    for (int c = 0; c < n_chunks; ++c) order[c] = c;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return delta[a] > delta[b]; });   // ties keep index order
+    std::vector<uint8_t> two(n_dft, 0);
+    for (int i = 0; i < n_keep; ++i) {
+        int lo, hi;
+        faedkv_chunk_range(n_dft, n_chunks, order[i], &lo, &hi);
+        std::fill(two.begin() + lo, two.begin() + hi, (uint8_t)1);
+    }
+    for (int k = 0; k <= n_dft / 2; ++k) mask_out[k] = (two[k] | two[(n_dft - k) % n_dft]) ? 1 : 0;
+    if (n_keep_out != nullptr) *n_keep_out = n_keep;
+    return FAEDKV_OK;
+}
+
+int faedkv_ablate(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch, int T, const float *gain,
+                  float *wsK, float *wsV, int32_t *ws_len, void *K_out, void *V_out, void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    if (K == nullptr || V == nullptr || gain == nullptr || wsK == nullptr || wsV == nullptr || ws_len == nullptr ||
+        K_out == nullptr || V_out == nullptr)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_ablate");
+    if (T < 1 || T > ctx->cfg.n_dft) return fail(ctx, FAEDKV_ERR_SHAPE, "T = %d outside [1, P=%d]", T, ctx->cfg.n_dft);
+    if (int r = check_ptrs(ctx, {K, V, gain, wsK, wsV, K_out, V_out})) return r;
+    if (int r = check_tlen(ctx, ws_len)) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const faedkv_config &c = ctx->cfg;
+    // spectrum of the touched bins, weighted by the share of each that the zeroing removes ...
+    if (int r = faedkv_compress_prefill(ctx, layer, K, V, batch, T, wsK, wsV, ws_len, stream)) return r;
+    const size_t n_vec = (size_t)batch * c.n_kv_heads * 2 * p->M * (kHeadDim / 4);
+    for (float *ws : {wsK, wsV}) {
+        k_scale_planes<<<(unsigned)((n_vec + 255) / 256), 256, 0, st>>>(ws, gain, p->M, n_vec);
+        if (int r = launch_check(ctx, "k_scale_planes")) return r;
+    }
+    // ... back to the time domain, and out of the input
+    if (int r = faedkv_reconstruct(ctx, layer, wsK, wsV, ws_len, batch, T, K_out, V_out, stream)) return r;
+    const size_t n = (size_t)batch * c.n_kv_heads * T * kHeadDim;
+    const void *xs[2] = {K, V};
+    void *ys[2] = {K_out, V_out};
+    for (int i = 0; i < 2; ++i) {
+        if (c.kv_dtype == FAEDKV_BF16)
+            k_subtract_from<__nv_bfloat16><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(xs[i]),
+                                                                                     static_cast<__nv_bfloat16 *>(ys[i]), n);
+        else
+            k_subtract_from<float><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(static_cast<const float *>(xs[i]),
+                                                                             static_cast<float *>(ys[i]), n);
+        if (int r = launch_check(ctx, "k_subtract_from")) return r;
+    }
+    return FAEDKV_OK;
 }
 
 unsigned long long faedkv_launch_count(const faedkv_ctx *ctx) { return ctx ? ctx->launches : 0ULL; }

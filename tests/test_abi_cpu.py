@@ -77,3 +77,28 @@ def test_create_rejects_bad_configs_before_touching_cuda(lib):
         assert not h.value
     assert lib.faedkv_create(None, ctypes.byref(h)) == -1
     lib.faedkv_destroy(None)  # allowed
+
+
+def test_selection_tooling_matches_the_oracle_bit_for_bit(lib, oracle):
+    """Chunk ranges, ablation bins / gains and the greedy keep-mask: host-only integer logic, identical to
+    the oracle's independent Python restatement."""
+    import numpy as np
+    from paper_2507_20030_b200 import binding
+    rng = np.random.default_rng(3)
+    for P, C in [(64, 22), (2048, 22), (100, 7), (32768, 22)]:
+        for c in range(C):
+            assert binding.chunk_range(P, C, c) == oracle.chunk_range(P, C, c)
+        for c in (0, 1, C // 2, C - 1):
+            lo, hi = oracle.chunk_range(P, C, c)
+            m, g = binding.ablation_bins(P, lo, hi)
+            om, og = oracle.ablation_bins(P, lo, hi)
+            assert m.tobytes() == om.tobytes() and g.tobytes() == og.tobytes()
+        for ratio in (0.05, 0.094, 0.125, 0.25, 1.0):
+            delta = np.round(rng.standard_normal(C), 1)             # rounded: ties occur
+            m, n = binding.mask_from_scores(P, C, delta, ratio)
+            om, on = oracle.mask_from_scores(P, C, delta, ratio)
+            assert n == on and m.tobytes() == om.tobytes(), (P, C, ratio)
+    with pytest.raises(binding.FaedkvError):
+        binding.chunk_range(64, 22, 22)
+    with pytest.raises(binding.FaedkvError):
+        binding.ablation_bins(64, 10, 10)

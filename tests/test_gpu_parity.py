@@ -592,3 +592,36 @@ def test_windowed_rejects_short_prefill_and_non_fft_grids(fk):
         ctx.step_windowed(0, x, x, x, cK, cK, w, w, t, x.clone())
     assert e.value.code == -4                                   # P = 100 has no FFT-shaped path
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- frequency ablation
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,T,C,chunks,B,H", [(1024, 1024, 22, (0, 3, 11, 21), 1, 2), (100, 100, 7, (0, 3, 6), 2, 1),
+                                              (256, 200, 22, (5, 10), 1, 3)])
+def test_ablate_matches_oracle(fk, oracle, dtype, P, T, C, chunks, B, H):
+    """Zeroing one chunk of the two-sided spectrum of K and V (Eq. 6), inverse transform, real part:
+    the removed component against the oracle's FFT definition."""
+    ctx = fk.Context(n_layers=len(chunks), n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype))
+    K, V = _make(61 + P, B, H, T, dtype)
+    for layer, c in enumerate(chunks):
+        lo, hi = fk.chunk_range(P, C, c)
+        mask, gain = fk.ablation_bins(P, lo, hi)
+        ctx.plan(layer, mask)
+        g = torch.from_numpy(gain[ctx.get_bins(layer)]).cuda()
+        wsK, wsV = ctx.alloc_coef(layer, B), ctx.alloc_coef(layer, B)
+        ws_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+        Ko = torch.full((B, H, T, 128), float("nan"), dtype=dtype, device="cuda")
+        Vo = torch.full_like(Ko, float("nan"))
+        ctx.ablate(layer, K.cuda(), V.cuda(), g, wsK, wsV, ws_len, Ko, Vo)
+        torch.cuda.synchronize()
+        assert ctx.device_status() == 0
+        for X, Xo in ((K, Ko), (V, Vo)):
+            x = to_np64(X)
+            want = np.stack([[oracle.ablate(x[b, h], P, lo, hi) for h in range(H)] for b in range(B)])
+            got = to_np64(Xo)
+            if dtype == torch.float32:
+                # compare what was removed: x' is close to x, so an error relative to x' would hide it
+                assert rel_l2(x - got, x - want) <= REL_L2_F32, (c, rel_l2(x - got, x - want))
+            else:
+                assert rel_l2(got, want) <= REL_L2_BF16, (c, rel_l2(got, want))
+    ctx.close()

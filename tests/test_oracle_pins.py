@@ -463,3 +463,56 @@ def test_windowed_folds_the_token_that_leaves_the_window(oracle):
     re, im = oracle.compress(K[S:t - R], P, bins)
     assert np.abs(u.CK[0] - re).max() < 1e-11 and np.abs(u.CK[1] - im).max() < 1e-11
     assert np.array_equal(np.stack(u.recentV), V[t - R:t]) and np.array_equal(u.sinkK, K[:S])
+
+
+# ----------------------------------------------------------------------------- ablation and selection
+def test_chunk_ranges_partition_the_grid(oracle):
+    for P, C in [(64, 22), (100, 7), (2048, 22), (22, 22)]:
+        edges = [oracle.chunk_range(P, C, c) for c in range(C)]
+        assert edges[0][0] == 0 and edges[-1][1] == P
+        assert all(edges[i][1] == edges[i + 1][0] for i in range(C - 1))
+        assert all(hi - lo == P // C for lo, hi in edges[:-1]) and edges[-1][1] - edges[-1][0] >= P // C
+
+
+@pytest.mark.parametrize("P,T,lo,hi", [(64, 64, 5, 9), (64, 64, 0, 3), (64, 64, 30, 35), (64, 64, 58, 64),
+                                       (96, 70, 40, 56), (33, 33, 10, 20)])
+def test_ablation_equals_removing_the_one_sided_components(oracle, P, T, lo, hi):
+    """The FFT definition of the ablation (zero two-sided bins, inverse, real part) against a second,
+    structurally different evaluation: x minus the gain-weighted reconstruction of the touched one-sided
+    bins by the C oracle's loops.  Pins the mirror bookkeeping (gain 1/2 when only one of k, P-k goes)."""
+    rng = np.random.default_rng(P + lo)
+    x = rng.standard_normal((T, 5))
+    want = oracle.ablate(x, P, lo, hi)
+    mask, gain = oracle.ablation_bins(P, lo, hi)
+    bins = oracle.plan(P, mask)
+    re, im = oracle.compress(x, P, bins)
+    g = gain[bins].astype(np.float64)[:, None]
+    removed = oracle.reconstruct(re * g, im * g, P, bins, T)
+    assert np.abs((x - removed) - want).max() < 1e-12
+    # a range that is its own mirror image removes whole conjugate pairs: the energy drops by exactly
+    # their share (Parseval), and the gains are all 1
+    if T == P and lo + (hi - 1) == P:
+        X = np.fft.fft(x, axis=0)
+        drop = (np.abs(X[lo:hi]) ** 2).sum() / P
+        assert abs(((x ** 2).sum() - (want ** 2).sum()) - drop) < 1e-9
+        assert (gain[bins] == 1.0).all()
+    else:
+        assert (gain[bins] == 0.5).any()
+
+
+def test_greedy_selection_rules(oracle):
+    P, C = 220, 22
+    delta = np.arange(C, dtype=np.float64)
+    delta[[3, 7]] = 100.0                      # a tie at the top: chunk 3 before chunk 7
+    mask, n_keep = oracle.mask_from_scores(P, C, delta, 0.125)          # 2.75 -> 3 chunks
+    assert n_keep == 3
+    kept2 = np.zeros(P, dtype=np.uint8)
+    for c in (3, 7, 21):
+        lo, hi = oracle.chunk_range(P, C, c)
+        kept2[lo:hi] = 1
+    assert mask.tobytes() == oracle.fold_two_sided(P, kept2).tobytes()
+    assert oracle.mask_from_scores(P, C, delta, 0.001)[1] == 1          # never fewer than one chunk
+    assert oracle.mask_from_scores(P, C, delta, 0.0682)[1] == 2         # 1.5004 rounds half up
+    m1, _ = oracle.mask_from_scores(P, C, np.zeros(C), 0.094)           # all tied: the lowest chunks win
+    lo, hi = oracle.chunk_range(P, C, 0)
+    assert m1[lo:hi].all() and m1[0] == 1
