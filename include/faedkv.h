@@ -254,6 +254,20 @@ int faedkv_ablate(faedkv_ctx *ctx, int layer, const void *K, const void *V, int 
                   const float *gain, float *wsK, float *wsV, int32_t *ws_len, void *K_out, void *V_out,
                   void *stream);
 
+/* ---- the state in the forms the paper's equations print (Sec. 4.1) ---------------------------------
+ * Every call of this library keeps the unnormalised, start-referenced sum
+ *   SUM       C_t[k] = sum_{n<t} x[n] exp(-j*2*pi*k*n/P).
+ * Eq. 9 with its exact factors (t-1)/t and 1/t keeps the running mean, and Eq. 8 / Eq. 9 as recursions
+ * that multiply the whole state by W_k = exp(-j*2*pi*k/P) each step keep a newest-token-referenced state:
+ *   MEAN      S_t[k] = C_t[k] / t
+ *   ROTATING  R_t[k] = W_k^t * conj(C_t[k])          (R <- W_k (R + x) from R_0 = 0)
+ * For real K/V the three hold the same information; this call converts a coefficient tensor between
+ * them, for exchanging state with an implementation that follows the printed recursions.  t = t_len[b];
+ * coef_in and coef_out have the coefficient layout and may be the same buffer. */
+typedef enum { FAEDKV_STATE_SUM = 0, FAEDKV_STATE_MEAN = 1, FAEDKV_STATE_ROTATING = 2 } faedkv_state_form;
+int faedkv_convert_state(faedkv_ctx *ctx, int layer, const float *coef_in, const int32_t *t_len,
+                         int batch, int from_form, int to_form, float *coef_out, void *stream);
+
 /* Device-side status word of the context (host read; synchronises `stream`):
  * 0, or a nonzero code left by a kernel whose bounded wait on an mbarrier gave
  * up.  Such a kernel returns early instead of hanging; its output is invalid. */

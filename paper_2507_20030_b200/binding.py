@@ -21,6 +21,7 @@ LIB_PATH = os.path.join(_HERE, "lib", "libfaedkv.so")
 
 F32, BF16 = 0, 1
 PREFILL_AUTO, PREFILL_SIMT, PREFILL_UMMA, PREFILL_FFT = 0, 1, 2, 3
+STATE_SUM, STATE_MEAN, STATE_ROTATING = 0, 1, 2
 DECODE_AUTO, DECODE_SIMT, DECODE_UMMA, DECODE_FFT = 0, 1, 2, 3
 
 EXPORTS = [
@@ -28,7 +29,7 @@ EXPORTS = [
     "faedkv_get_bins", "faedkv_coef_bytes", "faedkv_mask_lowpass", "faedkv_mask_mixed",
     "faedkv_compress_prefill", "faedkv_append", "faedkv_reconstruct", "faedkv_decode_attn",
     "faedkv_append_decode_attn", "faedkv_chunk_range", "faedkv_ablation_bins", "faedkv_mask_from_scores", "faedkv_ablate",
-    "faedkv_window_bytes", "faedkv_prefill_windowed", "faedkv_step_windowed",
+    "faedkv_convert_state", "faedkv_window_bytes", "faedkv_prefill_windowed", "faedkv_step_windowed",
     "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
 ]
 
@@ -98,6 +99,8 @@ def load() -> ctypes.CDLL:
     lib.faedkv_mask_from_scores.restype = _int
     lib.faedkv_ablate.argtypes = [_vp, _int, _vp, _vp, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
     lib.faedkv_ablate.restype = _int
+    lib.faedkv_convert_state.argtypes = [_vp, _int, _vp, _vp, _int, _int, _int, _vp, _vp]
+    lib.faedkv_convert_state.restype = _int
     lib.faedkv_window_bytes.argtypes = [_vp, _int]
     lib.faedkv_window_bytes.restype = ctypes.c_size_t
     lib.faedkv_prefill_windowed.argtypes = [_vp, _int, _vp, _vp, _int, _int, _vp, _vp, _vp, _vp, _vp, _vp]
@@ -305,6 +308,14 @@ class Context:
         self._check(self._lib.faedkv_ablate(
             self._h, layer, _ptr(K), _ptr(V), batch, T, _ptr(gain), _ptr(wsK), _ptr(wsV), _ptr(ws_len),
             _ptr(K_out), _ptr(V_out), _stream(stream)))
+
+    def convert_state(self, layer, coef_in, t_len, from_form, to_form, coef_out=None, stream=None):
+        """Stationary sum <-> running mean <-> rotating frame; in place when coef_out is None."""
+        coef_out = coef_in if coef_out is None else coef_out
+        self._check(self._lib.faedkv_convert_state(
+            self._h, layer, _ptr(coef_in), _ptr(t_len), t_len.shape[0], from_form, to_form, _ptr(coef_out),
+            _stream(stream)))
+        return coef_out
 
     # -- sink + recent window
     def alloc_window(self, batch: int, device="cuda") -> torch.Tensor:

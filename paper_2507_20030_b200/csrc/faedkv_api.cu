@@ -21,6 +21,7 @@
 #include "k_recon_fft.cuh"
 #include "k_prefill_fft.cuh"
 #include "k_ablate.cuh"
+#include "k_state.cuh"
 
 using namespace faedkv;
 
@@ -1194,6 +1195,25 @@ int faedkv_ablate(faedkv_ctx *ctx, int layer, const void *K, const void *V, int 
         if (int r = launch_check(ctx, "k_subtract_from")) return r;
     }
     return FAEDKV_OK;
+}
+
+int faedkv_convert_state(faedkv_ctx *ctx, int layer, const float *coef_in, const int32_t *t_len, int batch, int from_form,
+                         int to_form, float *coef_out, void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    if (coef_in == nullptr || coef_out == nullptr || t_len == nullptr)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_convert_state");
+    if (from_form < FAEDKV_STATE_SUM || from_form > FAEDKV_STATE_ROTATING || to_form < FAEDKV_STATE_SUM ||
+        to_form > FAEDKV_STATE_ROTATING)
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "unknown state form");
+    if (int r = check_ptrs(ctx, {coef_in, coef_out})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    dim3 grid((p->M + 7) / 8, batch * ctx->cfg.n_kv_heads);
+    k_convert_state<<<grid, 256, 0, st>>>(coef_in, coef_out, p->d_bins, t_len, p->M, ctx->cfg.n_kv_heads,
+                                          (uint32_t)ctx->cfg.n_dft, from_form, to_form);
+    return launch_check(ctx, "k_convert_state");
 }
 
 unsigned long long faedkv_launch_count(const faedkv_ctx *ctx) { return ctx ? ctx->launches : 0ULL; }

@@ -625,3 +625,41 @@ def test_ablate_matches_oracle(fk, oracle, dtype, P, T, C, chunks, B, H):
             else:
                 assert rel_l2(got, want) <= REL_L2_BF16, (c, rel_l2(got, want))
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- paper-literal state forms
+@pytest.mark.parametrize("P,T,M,B,H", [(64, 50, 9, 2, 2), (100, 230, 21, 1, 3)])
+def test_state_forms_match_the_printed_recursions(fk, oracle, P, T, M, B, H):
+    """The library's state converted to the rotating frame equals the oracle running the recursion
+    R <- W_k (R + x) literally over the tokens; converted to the running mean it equals the oracle's
+    exact-factor recursion; both conversions come back bit-close to the original."""
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=fk.F32,
+                     prefill_mode=fk.PREFILL_SIMT)
+    mask = _random_mask(P, M, 17 * P + T)
+    mask[0] = 1
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    M = len(bins)
+    K, V = _make(71 + P, B, H, T, torch.float32)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    rot = ctx.convert_state(0, cK, t_len, fk.STATE_SUM, fk.STATE_ROTATING, torch.empty_like(cK))
+    mean = ctx.convert_state(0, cK, t_len, fk.STATE_SUM, fk.STATE_MEAN, torch.empty_like(cK))
+    back1 = ctx.convert_state(0, rot.clone(), t_len, fk.STATE_ROTATING, fk.STATE_SUM)
+    back2 = ctx.convert_state(0, mean.clone(), t_len, fk.STATE_MEAN, fk.STATE_SUM)
+    cross = ctx.convert_state(0, rot.clone(), t_len, fk.STATE_ROTATING, fk.STATE_MEAN)
+    torch.cuda.synchronize()
+    x = to_np64(K)
+    for b in range(B):
+        for h in range(H):
+            Rre, Rim = np.zeros((M, 128)), np.zeros((M, 128))
+            Sre, Sim = np.zeros((M, 128)), np.zeros((M, 128))
+            for n in range(T):
+                oracle.rotating_frame_step(Rre, Rim, P, bins, x[b, h, n])
+                oracle.running_mean_step(Sre, Sim, P, bins, n, x[b, h, n])
+            assert rel_l2(to_np64(rot[b, h]), np.stack([Rre, Rim])) <= REL_L2_F32
+            assert rel_l2(to_np64(mean[b, h]), np.stack([Sre, Sim])) <= REL_L2_F32
+            assert rel_l2(to_np64(cross[b, h]), np.stack([Sre, Sim])) <= REL_L2_F32
+    assert rel_l2(to_np64(back1), to_np64(cK)) <= 1e-6 and rel_l2(to_np64(back2), to_np64(cK)) <= 1e-6
+    ctx.close()
