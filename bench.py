@@ -60,6 +60,25 @@ def _peaks():
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
 
 
+# --------------------------------------------------------------------------------------- ranks
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks (every rank gets the result).  The path
+    needs no inter-GPU exchange; this one reduction only puts the slowest replica's time on the line."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_value(units_per_rank: float, world: int, ms: float) -> float:
+    """Weak scaling over independent replicas: every rank processes `units_per_rank` in `ms` (the maximum over
+    ranks), so the job's throughput is world * units_per_rank / time."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 # --------------------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
@@ -377,10 +396,7 @@ def run_ours(args):
     step_ms = t_start.elapsed_time(t_stop) / args.steps
     prefill_ms = phase_ms["prefill"]
 
-    if world > 1:
-        t = torch.tensor([prefill_ms, step_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        prefill_ms, step_ms = float(t[0]), float(t[1])
+    prefill_ms, step_ms = max_over_ranks([prefill_ms, step_ms], dev)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region
     e2e = None
@@ -431,11 +447,8 @@ def run_ours(args):
         barrier()
         wall_ms = (time.perf_counter() - t0) * 1e3 / k_e2e
         e2e_ms = max(a.elapsed_time(b) / k_e2e, wall_ms if world == 1 else 0.0)
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t[0])
-        e2e = {"value": world * B * T / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e_ms = max_over_ranks([e2e_ms], dev)[0]
+        e2e = {"value": whole_job_value(B * T, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
                "what": "phase A through the C ABI with pinned host K/V in and host coefficient planes out"}
         del hK, hV, hcK, hcV
@@ -460,16 +473,13 @@ def run_ours(args):
         b.record(stream)
         barrier()
         f_ms = a.elapsed_time(b) / args.steps
-        if world > 1:
-            t = torch.tensor([f_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            f_ms = float(t[0])
+        f_ms = max_over_ranks([f_ms], dev)[0]
         n_cols = 2 * B * H * D                                           # channels of K and V
         lgN = (P // 2).bit_length() - 1
         flop = 5.0 * (P // 2) * lgN * n_cols                             # 5 N log2 N per complex length-N FFT
         f_bytes = 2 * B * H * T * D * 2 + 2 * B * H * 2 * M * D * 4      # K/V in (bf16) + planes out (float32)
         peak_alu = 148 * 128 * 2 * 1.965e9 / 1e12                        # float32 FMA lanes x 2 x max SM clock
-        prefill_fft = {"value": world * B * T / (f_ms * 1e-3), "unit": UNIT, "ms_per_layer": f_ms / NL,
+        prefill_fft = {"value": whole_job_value(B * T, world, f_ms), "unit": UNIT, "ms_per_layer": f_ms / NL,
                        "speedup_vs_value_path": prefill_ms / f_ms, "precision": "float32 (rel. error ~1e-6)",
                        "roofline": {"bound": "alu", "achieved": flop / (f_ms / NL * 1e-3) / 1e12, "peak": peak_alu,
                                     "unit": "TFLOP/s", "frac": flop / (f_ms / NL * 1e-3) / 1e12 / peak_alu,
@@ -547,7 +557,7 @@ def run_ours(args):
         # the headline decode number is the streaming-decode workload's
         decode["decode_us_per_layer_step_configs1_shape"] = decode["decode_us_per_layer_step"]
         decode["decode_us_per_layer_step"] = decode_sections[0]["decode_us_per_layer_step"]
-    line = {"metric": METRIC, "value": world * B * T / (prefill_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+    line = {"metric": METRIC, "value": whole_job_value(B * T, world, prefill_ms), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": W["name"], "n_layers": NL, "n_kv_heads": H, "n_q_heads": HQ, "head_dim": D,
