@@ -419,6 +419,12 @@ int launch_attn_tc(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const flo
         default: break;                                                                     \
     }
 
+// The instance with compile-time tile indexing when the launch uses the tile shape it was built for,
+// else the instance that takes the shape at run time.
+#define FFT_PICK(KERNEL, LG, lg_t) ((lg_t) == fft::fast_lg_transforms(LG) ? KERNEL<LG, fft::fast_lg_transforms(LG)> : KERNEL<LG, -1>)
+#define FFT_PICK_T(KERNEL, LG, lg_t, T) \
+    ((lg_t) == fft::fast_lg_transforms(LG) ? KERNEL<LG, fft::fast_lg_transforms(LG), T> : KERNEL<LG, -1, T>)
+
 template <typename K>
 int fft_opt_in(faedkv_ctx *ctx, K kernel, size_t bytes, unsigned int &done_mask, int lg) {
     if (bytes <= 48 * 1024 || (done_mask >> lg) & 1u) return FAEDKV_OK;
@@ -445,8 +451,8 @@ int launch_reconstruct_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const flo
             const dim3 grid(g.N2 >> lgKT, col_blocks);
             const size_t smem = afft_smem_a(g.lgN1, lgKT, true);
 #define CALL(LG)                                                                                         \
-            rc = fft_opt_in(ctx, k_rfft_inv_a<LG>, smem, f.attr_mask[3], LG);                            \
-            if (rc == 0) k_rfft_inv_a<LG><<<grid, fft::kThreads, smem, st>>>(g, p.d_slot, coef, p.M, u0, f.Yr, lgKT)
+            rc = fft_opt_in(ctx, FFT_PICK(k_rfft_inv_a, LG, lgKT), smem, f.attr_mask[3], LG + ((lgKT) == fft::fast_lg_transforms(LG) ? 16 : 0));                            \
+            if (rc == 0) FFT_PICK(k_rfft_inv_a, LG, lgKT)<<<grid, fft::kThreads, smem, st>>>(g, p.d_slot, coef, p.M, u0, f.Yr, lgKT)
             FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
 #undef CALL
             if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
@@ -457,8 +463,8 @@ int launch_reconstruct_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const flo
             const dim3 grid(g.N1 >> lgMT, col_blocks);
             const size_t smem = rfft_smem_b(g.lgN2, lgMT);
 #define CALL(LG)                                                                                         \
-            rc = fft_opt_in(ctx, k_rfft_inv_b<LG, TOut>, smem, f.attr_mask[kOutKind], LG);               \
-            if (rc == 0) k_rfft_inv_b<LG, TOut><<<grid, fft::kThreads, smem, st>>>(g, f.Yr, t_len, c.n_kv_heads, u0, L, static_cast<TOut *>(out), lgMT)
+            rc = fft_opt_in(ctx, FFT_PICK_T(k_rfft_inv_b, LG, lgMT, TOut), smem, f.attr_mask[kOutKind], LG + ((lgMT) == fft::fast_lg_transforms(LG) ? 16 : 0));               \
+            if (rc == 0) FFT_PICK_T(k_rfft_inv_b, LG, lgMT, TOut)<<<grid, fft::kThreads, smem, st>>>(g, f.Yr, t_len, c.n_kv_heads, u0, L, static_cast<TOut *>(out), lgMT)
             FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
 #undef CALL
             if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
@@ -498,8 +504,8 @@ int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x
             const dim3 grid(g.N1 >> lgMT, col_blocks);
             const size_t smem = pfft_smem_a(g.lgN2, lgMT);
 #define CALL(LG)                                                                                         \
-            rc = fft_opt_in(ctx, k_pfft_fwd_a<LG, TIn>, smem, f.attr_mask[kInKind], LG);                 \
-            if (rc == 0) k_pfft_fwd_a<LG, TIn><<<grid, fft::kThreads, smem, st>>>(g, static_cast<const TIn *>(x), T, T_stride, u0, f.Yr, lgMT)
+            rc = fft_opt_in(ctx, FFT_PICK_T(k_pfft_fwd_a, LG, lgMT, TIn), smem, f.attr_mask[kInKind], LG + ((lgMT) == fft::fast_lg_transforms(LG) ? 16 : 0));                 \
+            if (rc == 0) FFT_PICK_T(k_pfft_fwd_a, LG, lgMT, TIn)<<<grid, fft::kThreads, smem, st>>>(g, static_cast<const TIn *>(x), T, T_stride, u0, f.Yr, lgMT)
             FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
 #undef CALL
             if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
@@ -510,8 +516,8 @@ int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x
             const dim3 grid(g.N2 >> lgKT, col_blocks);
             const size_t smem = pfft_smem_b(g.lgN1, lgKT);
 #define CALL(LG)                                                                                         \
-            rc = fft_opt_in(ctx, k_pfft_fwd_b<LG>, smem, f.attr_mask[8], LG);                            \
-            if (rc == 0) k_pfft_fwd_b<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Yr, f.Zr, lgKT)
+            rc = fft_opt_in(ctx, FFT_PICK(k_pfft_fwd_b, LG, lgKT), smem, f.attr_mask[8], LG + ((lgKT) == fft::fast_lg_transforms(LG) ? 16 : 0));                            \
+            if (rc == 0) FFT_PICK(k_pfft_fwd_b, LG, lgKT)<<<grid, fft::kThreads, smem, st>>>(g, f.Yr, f.Zr, lgKT)
             FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
 #undef CALL
             if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
@@ -568,8 +574,8 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const dim3 grid(g.N2 >> lgKT, col_blocks);
         const size_t smem = afft_smem_a(g.lgN1, lgKT, true);
 #define CALL(LG)                                                                                         \
-        rc = fft_opt_in(ctx, k_afft_inv_a<LG>, smem, f.attr_mask[0], LG);                                \
-        if (rc == 0) k_afft_inv_a<LG><<<grid, fft::kThreads, smem, st>>>(g, p.d_slot, f.Qs, f.Y, lgKT)
+        rc = fft_opt_in(ctx, FFT_PICK(k_afft_inv_a, LG, lgKT), smem, f.attr_mask[0], LG + ((lgKT) == fft::fast_lg_transforms(LG) ? 16 : 0));                                \
+        if (rc == 0) FFT_PICK(k_afft_inv_a, LG, lgKT)<<<grid, fft::kThreads, smem, st>>>(g, p.d_slot, f.Qs, f.Y, lgKT)
         FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
@@ -580,8 +586,8 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const dim3 grid(g.N1 >> lgMT, col_blocks);
         const size_t smem = afft_smem_mid(g.lgN2, lgMT);
 #define CALL(LG)                                                                                         \
-        rc = fft_opt_in(ctx, k_afft_mid<LG>, smem, f.attr_mask[1], LG);                                  \
-        if (rc == 0) k_afft_mid<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Y, t_len, HQ, (APPEND ? 1 : 0) - S - R, f.mloc, f.sloc, lgMT)
+        rc = fft_opt_in(ctx, FFT_PICK(k_afft_mid, LG, lgMT), smem, f.attr_mask[1], LG + ((lgMT) == fft::fast_lg_transforms(LG) ? 16 : 0));                                  \
+        if (rc == 0) FFT_PICK(k_afft_mid, LG, lgMT)<<<grid, fft::kThreads, smem, st>>>(g, f.Y, t_len, HQ, (APPEND ? 1 : 0) - S - R, f.mloc, f.sloc, lgMT)
         FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
@@ -592,8 +598,8 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const dim3 grid(g.N2 >> lgKT, col_blocks);
         const size_t smem = afft_smem_fwd_b(g.lgN1, lgKT, lgMT);
 #define CALL(LG)                                                                                         \
-        rc = fft_opt_in(ctx, k_afft_fwd_b<LG>, smem, f.attr_mask[2], LG);                                \
-        if (rc == 0) k_afft_fwd_b<LG><<<grid, fft::kThreads, smem, st>>>(g, f.Y, f.mloc, f.sloc, lgMT, f.Zf, f.colsum, lgKT, n_extra)
+        rc = fft_opt_in(ctx, FFT_PICK(k_afft_fwd_b, LG, lgKT), smem, f.attr_mask[2], LG + ((lgKT) == fft::fast_lg_transforms(LG) ? 16 : 0));                                \
+        if (rc == 0) FFT_PICK(k_afft_fwd_b, LG, lgKT)<<<grid, fft::kThreads, smem, st>>>(g, f.Y, f.mloc, f.sloc, lgMT, f.Zf, f.colsum, lgKT, n_extra)
         FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;

@@ -92,10 +92,11 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
 // ---- (2) pass A of the inverse transform, half-spectrum packing fused into the load ----------------
 // slot[k], k in [0, N]: index of one-sided bin k in the plan, or -1.  Y: [N1][N2][Gp].
 // grid = (N2 / KT, Gp / 16); block = 256; dynamic smem = afft_smem_a(lgN1, lgKT, true).
-template <int LG>
+template <int LG, int LGT>
 __global__ void __launch_bounds__(fft::kThreads)
 k_afft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float2 *__restrict__ Qs,
-             float2 *__restrict__ Y, int lgKT) {
+             float2 *__restrict__ Y, int lgKT_rt) {
+    const int lgKT = LGT >= 0 ? LGT : lgKT_rt;   // compile-time in the fast instances
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N1
     extern __shared__ float2 fft_smem[];
@@ -132,17 +133,18 @@ k_afft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float2 *__
         const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
         Y[y_index(g, m1, k2_0 + kt, g0 + c)] = cmul(v, tab_i[(m1 << lgKT) + kt]);
     };
-    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+    fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
 }
 
 // ---- pass B of the inverse transform, local softmax, pass A' of the forward transform ---------------
 // One CTA = MT values of m1 (one "tile" of the softmax statistics) x 16 columns.
 // mloc, sloc: [N1 / MT][Gp].  live length of a column = min(t_len[col / HQ] + t_add, P).
 // grid = (N1 / MT, Gp / 16); block = 256; dynamic smem = afft_smem_mid(lgN2, lgMT).
-template <int LG>
+template <int LG, int LGT>
 __global__ void __launch_bounds__(fft::kThreads)
 k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ t_len, int HQ, int t_add,
-           float *__restrict__ mloc, float *__restrict__ sloc, int lgMT) {
+           float *__restrict__ mloc, float *__restrict__ sloc, int lgMT_rt) {
+    const int lgMT = LGT >= 0 ? LGT : lgMT_rt;   // compile-time in the fast instances
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N2
     extern __shared__ float2 fft_smem[];
@@ -176,7 +178,7 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
             return Y[y_index(g, m1_0 + (cidx >> kLgCW), k2, g0 + (cidx & (kCW - 1)))];
         };
         auto store = [&](int m2, int cidx, float2 v) { T[(m2 << lg_cols) + cidx] = v; };
-        fft_rows<LG>(lg_cols, xa, xb, tw, load, store);      // T[m2][mt, c] = z[m1 + N1 m2]
+        fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);      // T[m2][mt, c] = z[m1 + N1 m2]
     }
     __syncthreads();
     // a thread always meets the same column: kThreads is a multiple of 16
@@ -225,7 +227,7 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
             const int mt = cidx >> kLgCW;
             Y[y_index(g, m1_0 + mt, k1p, g0 + (cidx & (kCW - 1)))] = cmul(v, tab_i[(k1p << lgMT) + mt]);
         };
-        fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+        fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
     }
 }
 
@@ -234,11 +236,12 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
 // The CTAs with blockIdx.x == 0 also write the softmax normaliser colsum[col] = sum_tiles sloc * factor.
 // Zf: [N][Gp], index k1' + N2 * k2'.
 // grid = (N2 / KT, Gp / 16); block = 256; dynamic smem = afft_smem_a(lgN1, lgKT, false) + factors.
-template <int LG>
+template <int LG, int LGT>
 __global__ void __launch_bounds__(fft::kThreads)
 k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restrict__ mloc,
-             const float *__restrict__ sloc, int lgMT, float2 *__restrict__ Zf, float *__restrict__ colsum, int lgKT,
+             const float *__restrict__ sloc, int lgMT, float2 *__restrict__ Zf, float *__restrict__ colsum, int lgKT_rt,
              int n_extra) {
+    const int lgKT = LGT >= 0 ? LGT : lgKT_rt;   // compile-time in the fast instances
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N1
     extern __shared__ float2 fft_smem[];
@@ -301,7 +304,7 @@ k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restr
     auto store = [&](int k2p, int cidx, float2 v) {
         Zf[((uint32_t)(k1_0 + (cidx >> kLgCW)) + (uint32_t)g.N2 * (uint32_t)k2p) * (uint32_t)g.Gp + (uint32_t)(g0 + (cidx & (kCW - 1)))] = v;
     };
-    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+    fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
 }
 
 // Dynamic shared memory of the three kernels above (bytes).

@@ -149,10 +149,14 @@ __host__ __device__ constexpr int exchange_buffers(int lg) { return lg >= 9 ? 2 
 
 // One Stockham stage of radix R over NF rows x (1 << lg_cols) columns; NS = product of the radices
 // already applied.  in(row, col) -> float2, out(row, col, value).
-template <int NF, int R, int NS, typename In, typename Out>
-__device__ __forceinline__ void fft_stage(int lg_cols, const float2 *__restrict__ tw, In in, Out out) {
+// LGC >= 0 fixes lg_cols at compile time (index arithmetic then folds into constants: these kernels are bound
+// by integer ALU work, not by the butterflies); LGC = -1 takes the run-time value.
+template <int NF, int R, int NS, int LGC, typename In, typename Out>
+__device__ __forceinline__ void fft_stage(int lg_cols_rt, const float2 *__restrict__ tw, In in, Out out) {
     constexpr int NB = NF / R;          // butterflies per column; also the row stride of a butterfly's inputs
+    const int lg_cols = LGC >= 0 ? LGC : lg_cols_rt;
     const int items = NB << lg_cols;
+#pragma unroll
     for (int it = threadIdx.x; it < items; it += kThreads) {
         const int c = it & ((1 << lg_cols) - 1), j = it >> lg_cols;
         float2 v[R];
@@ -174,28 +178,33 @@ __device__ __forceinline__ void fft_stage(int lg_cols, const float2 *__restrict_
 // inputs, store(row, col, value) takes the outputs; xa, xb are the exchange buffers (see
 // exchange_buffers()), tw the NF-entry twiddle table.  All threads of the CTA must call it; it
 // contains __syncthreads() between stages but none before the first or after the last stage.
-template <int LG, typename Load, typename Store>
-__device__ __forceinline__ void fft_rows(int lg_cols, float2 *xa, float2 *xb, const float2 *tw, Load load, Store store) {
+template <int LG, int LGC, typename Load, typename Store>
+__device__ __forceinline__ void fft_rows(int lg_cols_rt, float2 *xa, float2 *xb, const float2 *tw, Load load, Store store) {
     constexpr int NF = 1 << LG;
+    const int lg_cols = LGC >= 0 ? LGC : lg_cols_rt;
     constexpr int R1 = Radix<LG>::R1, R2 = Radix<LG>::R2, R3 = Radix<LG>::R3;
     auto rd_a = [&](int row, int c) { return xa[(row << lg_cols) + c]; };
     auto wr_a = [&](int row, int c, float2 v) { xa[(row << lg_cols) + c] = v; };
     auto rd_b = [&](int row, int c) { return xb[(row << lg_cols) + c]; };
     auto wr_b = [&](int row, int c, float2 v) { xb[(row << lg_cols) + c] = v; };
     if constexpr (R2 == 1) {
-        fft_stage<NF, R1, 1>(lg_cols, tw, load, store);
+        fft_stage<NF, R1, 1, LGC>(lg_cols, tw, load, store);
     } else if constexpr (R3 == 1) {
-        fft_stage<NF, R1, 1>(lg_cols, tw, load, wr_a);
+        fft_stage<NF, R1, 1, LGC>(lg_cols, tw, load, wr_a);
         __syncthreads();
-        fft_stage<NF, R2, R1>(lg_cols, tw, rd_a, store);
+        fft_stage<NF, R2, R1, LGC>(lg_cols, tw, rd_a, store);
     } else {
-        fft_stage<NF, R1, 1>(lg_cols, tw, load, wr_a);
+        fft_stage<NF, R1, 1, LGC>(lg_cols, tw, load, wr_a);
         __syncthreads();
-        fft_stage<NF, R2, R1>(lg_cols, tw, rd_a, wr_b);
+        fft_stage<NF, R2, R1, LGC>(lg_cols, tw, rd_a, wr_b);
         __syncthreads();
-        fft_stage<NF, R3, R1 * R2>(lg_cols, tw, rd_b, store);
+        fft_stage<NF, R3, R1 * R2, LGC>(lg_cols, tw, rd_b, store);
     }
 }
+
+// The number of transforms per CTA (lg) for which the kernels have a compile-time-indexed instance: a 4096-element
+// tile where the row count allows.
+__host__ __device__ constexpr int fast_lg_transforms(int lg_rows) { return lg_rows >= 8 ? 0 : (lg_rows == 7 ? 1 : 2); }
 
 // Element (m1, row, col) of the intermediate array between the two passes: [N1][N2][Gp] float2.
 // 32-bit on purpose (address arithmetic is a visible share of these kernels' instructions): the host

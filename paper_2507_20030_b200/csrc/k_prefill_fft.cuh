@@ -18,9 +18,10 @@
 namespace faedkv {
 
 // grid = (N1 / MT, cols / 16); block = 256.  x: rows of the tensor, T rows per unit, units T_stride rows apart.
-template <int LG, typename TIn>
+template <int LG, int LGT, typename TIn>
 __global__ void __launch_bounds__(fft::kThreads)
-k_pfft_fwd_a(fft::Geometry g, const TIn *__restrict__ x, int T, int T_stride, int unit0, float2 *__restrict__ U, int lgMT) {
+k_pfft_fwd_a(fft::Geometry g, const TIn *__restrict__ x, int T, int T_stride, int unit0, float2 *__restrict__ U, int lgMT_rt) {
+    const int lgMT = LGT >= 0 ? LGT : lgMT_rt;   // compile-time in the fast instances
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N2
     extern __shared__ float2 fft_smem[];
@@ -59,13 +60,14 @@ k_pfft_fwd_a(fft::Geometry g, const TIn *__restrict__ x, int T, int T_stride, in
         const int mt = cidx >> kLgCW;
         U[y_index(g, m1_0 + mt, k1p, g0 + (cidx & (kCW - 1)))] = cmul(v, tab_i[(k1p << lgMT) + mt]);
     };
-    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+    fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
 }
 
 // grid = (N2 / KT, cols / 16); block = 256.
-template <int LG>
+template <int LG, int LGT>
 __global__ void __launch_bounds__(fft::kThreads)
-k_pfft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, float2 *__restrict__ Zf, int lgKT) {
+k_pfft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, float2 *__restrict__ Zf, int lgKT_rt) {
+    const int lgKT = LGT >= 0 ? LGT : lgKT_rt;   // compile-time in the fast instances
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N1
     extern __shared__ float2 fft_smem[];
@@ -81,7 +83,7 @@ k_pfft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, float2 *__restrict__
         Zf[((uint32_t)(k1_0 + (cidx >> kLgCW)) + (uint32_t)g.N2 * (uint32_t)k2p) * (uint32_t)g.Gp +
            (uint32_t)(g0 + (cidx & (kCW - 1)))] = v;
     };
-    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+    fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
 }
 
 // Coefficients at the retained bins.  grid = (ceil(M / 8), cols / 128); block = 256: a warp per bin,

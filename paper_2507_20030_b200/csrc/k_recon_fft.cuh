@@ -18,10 +18,11 @@ namespace faedkv {
 
 // grid = (N2 / KT, cols / 16); block = 256; dynamic smem as k_afft_inv_a.
 // coef: planes of the tensor, [units][2][M][128]; unit0: first unit of this launch.
-template <int LG>
+template <int LG, int LGT>
 __global__ void __launch_bounds__(fft::kThreads)
 k_rfft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float *__restrict__ coef, int M, int unit0,
-             float2 *__restrict__ Y, int lgKT) {
+             float2 *__restrict__ Y, int lgKT_rt) {
+    const int lgKT = LGT >= 0 ? LGT : lgKT_rt;   // compile-time in the fast instances
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N1
     extern __shared__ float2 fft_smem[];
@@ -63,15 +64,16 @@ k_rfft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float *__r
         const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
         Y[y_index(g, m1, k2_0 + kt, g0 + c)] = cmul(v, tab_i[(m1 << lgKT) + kt]);
     };
-    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+    fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
 }
 
 // grid = (N1 / MT, cols / 16); block = 256; dynamic smem = rfft_smem_b(lgN2, lgMT).
 // out: rows of the tensor, [units][Lrows][128]; H: kv heads per sequence (t_len index = unit / H).
-template <int LG, typename TOut>
+template <int LG, int LGT, typename TOut>
 __global__ void __launch_bounds__(fft::kThreads)
 k_rfft_inv_b(fft::Geometry g, const float2 *__restrict__ Y, const int32_t *__restrict__ t_len, int H, int unit0,
-             int Lrows, TOut *__restrict__ out, int lgMT) {
+             int Lrows, TOut *__restrict__ out, int lgMT_rt) {
+    const int lgMT = LGT >= 0 ? LGT : lgMT_rt;   // compile-time in the fast instances
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N2
     extern __shared__ float2 fft_smem[];
@@ -96,7 +98,7 @@ k_rfft_inv_b(fft::Geometry g, const float2 *__restrict__ Y, const int32_t *__res
         if (n < Lrows) store1(o, n < live ? v.x : 0.f);
         if (n + 1 < Lrows) store1(o + kHeadDim, n + 1 < live ? v.y : 0.f);
     };
-    fft_rows<LG>(lg_cols, xa, xb, tw, load, store);
+    fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
 }
 
 inline size_t rfft_smem_b(int lg, int lgMT) {
