@@ -60,6 +60,14 @@ __device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v) {
 __device__ __forceinline__ void store1(float *p, float v) { *p = v; }
 __device__ __forceinline__ void store1(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute is
+// scheduled while its predecessor in the stream drains, and runs its own set-up (tables in shared memory)
+// at once; it must call pdl_wait() before touching anything the predecessor writes -- the wait returns when
+// the predecessor has completed and its writes are visible.  Without the attribute it is a no-op.
+// (Letting the predecessor release its dependents early, by griddepcontrol.launch_dependents at its start,
+// was measured slower here: the waiting CTAs hold shared memory and registers the predecessor still needs.)
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Streaming (evict-first) 16-byte global accesses for planes that are touched
 // once per call and are far larger than L2.
 __device__ __forceinline__ float4 ld_stream(const float *p) {

@@ -425,6 +425,23 @@ int launch_attn_tc(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const flo
 #define FFT_PICK_T(KERNEL, LG, lg_t, T) \
     ((lg_t) == fft::fast_lg_transforms(LG) ? KERNEL<LG, fft::fast_lg_transforms(LG), T> : KERNEL<LG, -1, T>)
 
+// Launch with programmatic stream serialisation: the kernel may begin (up to its pdl_wait()) before the
+// previous kernel of the stream has finished.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <typename K>
 int fft_opt_in(faedkv_ctx *ctx, K kernel, size_t bytes, unsigned int &done_mask, int lg) {
     if (bytes <= 48 * 1024 || (done_mask >> lg) & 1u) return FAEDKV_OK;
@@ -575,7 +592,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const size_t smem = afft_smem_a(g.lgN1, lgKT, true);
 #define CALL(LG)                                                                                         \
         rc = fft_opt_in(ctx, FFT_PICK(k_afft_inv_a, LG, lgKT), smem, f.attr_mask[0], LG + ((lgKT) == fft::fast_lg_transforms(LG) ? 16 : 0));                                \
-        if (rc == 0) FFT_PICK(k_afft_inv_a, LG, lgKT)<<<grid, fft::kThreads, smem, st>>>(g, p.d_slot, f.Qs, f.Y, lgKT)
+        if (rc == 0) launch_pdl(FFT_PICK(k_afft_inv_a, LG, lgKT), grid, dim3(fft::kThreads), smem, st, g, p.d_slot, f.Qs, f.Y, lgKT)
         FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
@@ -587,7 +604,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const size_t smem = afft_smem_mid(g.lgN2, lgMT);
 #define CALL(LG)                                                                                         \
         rc = fft_opt_in(ctx, FFT_PICK(k_afft_mid, LG, lgMT), smem, f.attr_mask[1], LG + ((lgMT) == fft::fast_lg_transforms(LG) ? 16 : 0));                                  \
-        if (rc == 0) FFT_PICK(k_afft_mid, LG, lgMT)<<<grid, fft::kThreads, smem, st>>>(g, f.Y, t_len, HQ, (APPEND ? 1 : 0) - S - R, f.mloc, f.sloc, lgMT)
+        if (rc == 0) launch_pdl(FFT_PICK(k_afft_mid, LG, lgMT), grid, dim3(fft::kThreads), smem, st, g, f.Y, t_len, HQ, (APPEND ? 1 : 0) - S - R, f.mloc, f.sloc, lgMT)
         FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
@@ -599,7 +616,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const size_t smem = afft_smem_fwd_b(g.lgN1, lgKT, lgMT);
 #define CALL(LG)                                                                                         \
         rc = fft_opt_in(ctx, FFT_PICK(k_afft_fwd_b, LG, lgKT), smem, f.attr_mask[2], LG + ((lgKT) == fft::fast_lg_transforms(LG) ? 16 : 0));                                \
-        if (rc == 0) FFT_PICK(k_afft_fwd_b, LG, lgKT)<<<grid, fft::kThreads, smem, st>>>(g, f.Y, f.mloc, f.sloc, lgMT, f.Zf, f.colsum, lgKT, n_extra)
+        if (rc == 0) launch_pdl(FFT_PICK(k_afft_fwd_b, LG, lgKT), grid, dim3(fft::kThreads), smem, st, g, f.Y, f.mloc, f.sloc, lgMT, f.Zf, f.colsum, lgKT, n_extra)
         FAEDKV_FFT_SWITCH(g.lgN1, 3, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
@@ -609,9 +626,9 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const int slices = out_slices(ctx, batch, M);
         const int per = (M + slices - 1) / slices;
         dim3 grid(slices, batch * H);
-        k_attn_out_fft<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(
-            coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
-            static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, windowed ? 0 : 1);
+        launch_pdl(k_attn_out_fft<TQ, GQ, APPEND>, grid, dim3(kAttnWarps * 32), 0, st,
+                   coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
+                   static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, windowed ? 0 : 1);
         if (int r = launch_check(ctx, "k_attn_out_fft")) return r;
     }
     if (windowed) {

@@ -29,6 +29,7 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
           const int32_t *__restrict__ t_len, const int32_t *__restrict__ bins, float2 *__restrict__ Qs,
           int M, int H, int HQ, int Gp, uint32_t P, float scale_over_P, FoldSrc fold) {
     constexpr int KB = 16 / GQ;
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
     const int k0 = (blockIdx.x * kAttnWarps + warp) * KB;
@@ -115,7 +116,9 @@ k_afft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float2 *__
         tab_p[e] = unit_phasor((uint32_t)(g.N2 * r + k2_0 + kt), g.P);
         tab_s[e] = make_int2(slot[g.N2 * r + k2_0 + kt], slot[g.N - (g.N2 * r + k2_0 + kt)]);
     }
+
     __syncthreads();
+    pdl_wait();                                      // Qs comes from the previous kernel
     auto load = [&](int k1, int cidx) {
         const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
         const int col = g0 + c;
@@ -172,7 +175,9 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
         }
         live_s[threadIdx.x] = live;
     }
+
     __syncthreads();
+    pdl_wait();                                      // Y comes from the previous kernel
     {
         auto load = [&](int k2, int cidx) {
             return Y[y_index(g, m1_0 + (cidx >> kLgCW), k2, g0 + (cidx & (kCW - 1)))];
@@ -258,6 +263,8 @@ k_afft_fwd_b(fft::Geometry g, const float2 *__restrict__ U, const float *__restr
     // the softmax as one more tile; its factor is handed to the output kernel in colsum[Gp + col]
     const int n_stat = n_tiles + n_extra;
     fill_twiddles(tw, NF);
+
+    pdl_wait();                                      // the statistics and Y come from the previous kernel
     const int c = threadIdx.x & (kCW - 1);
     {
         float mx = -INFINITY;
@@ -364,6 +371,7 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
     float4 acc[GQ];
 #pragma unroll
     for (int q = 0; q < GQ; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    pdl_wait();                                      // Zf and the normalisers come from the previous kernel
 
     for (int c0 = kbeg; c0 < kend; c0 += kOutChunk) {
         const int cn = min(kOutChunk, kend - c0);

@@ -55,6 +55,7 @@ k_attn_window(const TQ *__restrict__ q, const TQ *__restrict__ winK, const TQ *_
               const TQ *__restrict__ k_new, const TQ *__restrict__ v_new, const int32_t *__restrict__ t_len, int H,
               int S, int R, float scale, float *__restrict__ m_w, float *__restrict__ s_w, float *__restrict__ o_w) {
     extern __shared__ float sc[];                     // [GQ][W]
+
     const int W = S + R;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.x, b = bh / H;
