@@ -85,17 +85,23 @@ __device__ __forceinline__ void fill_twiddles(float2 *tw, int NF) {
 
 // ---- register butterflies: DFT of size R with kernel e^{+j 2 pi kr / R} ----------------------------------
 // Output r of the DFT is left in v[perm<R>(r)] (identity except for R = 16).
+// Complex additions use the packed float32x2 instructions of sm_100 (one issue slot for both components;
+// these kernels are issue-bound and additions are their largest instruction class); a - b is the packed FMA
+// b * (-1) + a, which rounds exactly like the subtraction.  Rotations by +-j stay scalar: they only rename
+// components, which packed operands cannot do for free.
+__device__ __forceinline__ float2 padd(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float2 psub(float2 a, float2 b) { return __ffma2_rn(b, make_float2(-1.f, -1.f), a); }
 __device__ __forceinline__ void dft2(float2 &a, float2 &b) {
     const float2 t = a;
-    a = cadd(t, b);
-    b = csub(t, b);
+    a = padd(t, b);
+    b = psub(t, b);
 }
 __device__ __forceinline__ void dft4(float2 &v0, float2 &v1, float2 &v2, float2 &v3) {
-    const float2 a0 = cadd(v0, v2), a1 = csub(v0, v2), a2 = cadd(v1, v3), a3 = cmulj(csub(v1, v3));
-    v0 = cadd(a0, a2);
-    v1 = cadd(a1, a3);
-    v2 = csub(a0, a2);
-    v3 = csub(a1, a3);
+    const float2 a0 = padd(v0, v2), a1 = psub(v0, v2), a2 = padd(v1, v3), d = psub(v1, v3);
+    v0 = padd(a0, a2);
+    v2 = psub(a0, a2);
+    v1 = make_float2(a1.x - d.y, a1.y + d.x);        // a1 + j d
+    v3 = make_float2(a1.x + d.y, a1.y - d.x);        // a1 - j d
 }
 template <int R> __device__ __forceinline__ void dft(float2 (&v)[R]);
 template <> __device__ __forceinline__ void dft<2>(float2 (&v)[2]) { dft2(v[0], v[1]); }
@@ -106,13 +112,14 @@ template <> __device__ __forceinline__ void dft<8>(float2 (&v)[8]) {
     const float h = 0.70710678118654752f;
     const float2 o0 = v[1];
     const float2 o1 = make_float2(h * (v[3].x - v[3].y), h * (v[3].x + v[3].y));     // * e^{+j pi/4}
-    const float2 o2 = cmulj(v[5]);                                                    // * e^{+j pi/2}
+    const float2 o2 = v[5];                                                           // * e^{+j pi/2}, applied below
     const float2 o3 = make_float2(-h * (v[7].x + v[7].y), h * (v[7].x - v[7].y));    // * e^{+j 3pi/4}
     const float2 e0 = v[0], e1 = v[2], e2 = v[4], e3 = v[6];
-    v[0] = cadd(e0, o0); v[4] = csub(e0, o0);
-    v[1] = cadd(e1, o1); v[5] = csub(e1, o1);
-    v[2] = cadd(e2, o2); v[6] = csub(e2, o2);
-    v[3] = cadd(e3, o3); v[7] = csub(e3, o3);
+    v[0] = padd(e0, o0); v[4] = psub(e0, o0);
+    v[1] = padd(e1, o1); v[5] = psub(e1, o1);
+    v[2] = make_float2(e2.x - o2.y, e2.y + o2.x);    // e2 + j o2
+    v[6] = make_float2(e2.x + o2.y, e2.y - o2.x);    // e2 - j o2
+    v[3] = padd(e3, o3); v[7] = psub(e3, o3);
 }
 // 16 = 4 x 4: n = n1 + 4 n2, k = k2 + 4 k1; X[k2 + 4 k1] ends in v[k1 + 4 k2].
 template <> __device__ __forceinline__ void dft<16>(float2 (&v)[16]) {
