@@ -227,11 +227,11 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     # windows of the paper's workflow (sink 10 + recent 50), filled with tokens of the same distributions
     wK, wV = synth.make_kv(seed + 7, B, H, 60, D, pos0=T - 60, dtype=torch.bfloat16, device=dev)
     loops = {
-        "step_windowed": lambda: [ctx.step_windowed(l, k_new, v_new, q, cKs[l], cVs[l], wK, wV, tls[l], out) for l in range(NL)],
         "append": lambda: [ctx.append(l, k_new, v_new, cKs[l], cVs[l], tls[l]) for l in range(NL)],
         "decode_attn": lambda: [ctx.decode_attn(l, q, cKs[l], cVs[l], tls[l], out) for l in range(NL)],
         "append_decode_attn": lambda: [ctx.append_decode_attn(l, k_new, v_new, q, cKs[l], cVs[l], tls[l], out)
                                        for l in range(NL)],
+        "step_windowed": lambda: [ctx.step_windowed(l, k_new, v_new, q, cKs[l], cVs[l], wK, wV, tls[l], out) for l in range(NL)],
     }
     coef_bytes = 2 * B * H * 2 * M * D * 4                      # K and V planes of one layer
     alg_bytes = {"append": 2 * coef_bytes, "decode_attn": coef_bytes, "append_decode_attn": 2 * coef_bytes,

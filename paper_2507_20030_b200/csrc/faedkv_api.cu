@@ -52,6 +52,8 @@ struct FftScratch {
     int recon_units = 0;                  // units (sequence, kv head) per launch group of the reconstruction
     float *mloc = nullptr, *sloc = nullptr, *colsum = nullptr;   // [N1 + 1][Gp] (last row: the window), [2][Gp]
     float *o_win = nullptr;               // [Gp][128] unnormalised attention output over the sink + recent window
+    cudaStream_t side = nullptr;          // second stream: the window kernel runs beside the FFT kernels
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     unsigned int *tickets = nullptr;      // [max_batch * H + max_batch], zero between calls
     int max_M = 0;
     unsigned int attr_mask[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
@@ -160,6 +162,9 @@ void free_scratch(faedkv_ctx *ctx) {
     t = TcScratch();
     FftScratch &f = ctx->fs;
     cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.o_win); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr);
+    if (f.side != nullptr) cudaStreamDestroy(f.side);
+    if (f.ev_fork != nullptr) cudaEventDestroy(f.ev_fork);
+    if (f.ev_join != nullptr) cudaEventDestroy(f.ev_join);
     f = FftScratch();
 }
 
@@ -197,7 +202,12 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             CUDA_TRY(ctx, cudaMalloc(&f.mloc, (size_t)(g.N1 + 1) * g.Gp * sizeof(float)));
             CUDA_TRY(ctx, cudaMalloc(&f.sloc, (size_t)(g.N1 + 1) * g.Gp * sizeof(float)));
             CUDA_TRY(ctx, cudaMalloc(&f.colsum, (size_t)2 * g.Gp * sizeof(float)));
-            if (c.n_sink + c.n_recent > 0) CUDA_TRY(ctx, cudaMalloc(&f.o_win, (size_t)g.Gp * kHeadDim * sizeof(float)));
+            if (c.n_sink + c.n_recent > 0) {
+                CUDA_TRY(ctx, cudaMalloc(&f.o_win, (size_t)g.Gp * kHeadDim * sizeof(float)));
+                CUDA_TRY(ctx, cudaStreamCreateWithFlags(&f.side, cudaStreamNonBlocking));
+                CUDA_TRY(ctx, cudaEventCreateWithFlags(&f.ev_fork, cudaEventDisableTiming));
+                CUDA_TRY(ctx, cudaEventCreateWithFlags(&f.ev_join, cudaEventDisableTiming));
+            }
             const size_t n_tickets = (size_t)c.max_batch * c.n_kv_heads + c.max_batch;
             CUDA_TRY(ctx, cudaMalloc(&f.tickets, n_tickets * sizeof(unsigned int)));
             CUDA_TRY(ctx, cudaMemset(f.tickets, 0, n_tickets * sizeof(unsigned int)));
@@ -573,18 +583,23 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
     constexpr int KB = 16 / GQ;
     {
         dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
-        k_attn_qs<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(static_cast<const TQ *>(q), coefK,
-                                                                     static_cast<const TQ *>(foldK), t_len, p.d_bins, f.Qs, M, H,
-                                                                     HQ, g.Gp, (uint32_t)P, scale / (float)P, fold);
+        k_attn_qs<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(
+            static_cast<const TQ *>(q), coefK, static_cast<const TQ *>(foldK), t_len, p.d_bins, f.Qs, M, H, HQ, g.Gp,
+            (uint32_t)P, scale / (float)P, fold);
         if (int r = launch_check(ctx, "k_attn_qs")) return r;
     }
     if (n_extra) {
+        // the window's scores, statistics (one more "tile" row) and unnormalised output, on the context's
+        // second stream beside the next two kernels (which leave the memory system idle); joined before the
+        // kernel that reads the statistics
         const int n_tiles = g.N1 >> lgMT;
-        k_attn_window<TQ, GQ><<<batch * H, 256, (size_t)GQ * (S + R) * sizeof(float), st>>>(
-            static_cast<const TQ *>(q), static_cast<const TQ *>(winK), static_cast<const TQ *>(winV),
-            static_cast<const TQ *>(k_new), static_cast<const TQ *>(v_new), t_len, H, S, R, scale,
-            f.mloc + (size_t)n_tiles * g.Gp, f.sloc + (size_t)n_tiles * g.Gp, f.o_win);
+        const WindowArgs wa{winK, winV, k_new, v_new, S, R, scale, f.mloc + (size_t)n_tiles * g.Gp,
+                            f.sloc + (size_t)n_tiles * g.Gp, f.o_win};
+        CUDA_TRY(ctx, cudaEventRecord(f.ev_fork, st));
+        CUDA_TRY(ctx, cudaStreamWaitEvent(f.side, f.ev_fork, 0));
+        k_attn_window<TQ, GQ><<<dim3(batch * H, GQ), 256, (size_t)(S + R) * sizeof(float), f.side>>>(static_cast<const TQ *>(q), wa, t_len, H);
         if (int r = launch_check(ctx, "k_attn_window")) return r;
+        CUDA_TRY(ctx, cudaEventRecord(f.ev_join, f.side));
     }
     int rc = FAEDKV_ERR_UNSUPPORTED;
     {
@@ -610,6 +625,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
         if (int r = launch_check(ctx, "k_afft_mid")) return r;
     }
+    if (n_extra) CUDA_TRY(ctx, cudaStreamWaitEvent(st, f.ev_join, 0));
     rc = FAEDKV_ERR_UNSUPPORTED;
     {
         const dim3 grid(g.N2 >> lgKT, col_blocks);
@@ -628,13 +644,9 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         dim3 grid(slices, batch * H);
         launch_pdl(k_attn_out_fft<TQ, GQ, APPEND>, grid, dim3(kAttnWarps * 32), 0, st,
                    coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
-                   static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, windowed ? 0 : 1);
+                   static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, 1,
+                   windowed ? WindowArgs{winK, winV, k_new, v_new, S, R, 0.f, nullptr, nullptr, nullptr} : WindowArgs{});
         if (int r = launch_check(ctx, "k_attn_out_fft")) return r;
-    }
-    if (windowed) {
-        k_window_commit<TQ><<<batch, kHeadDim, 0, st>>>(static_cast<const TQ *>(k_new), static_cast<const TQ *>(v_new),
-                                                        static_cast<TQ *>(winK), static_cast<TQ *>(winV), t_len, H, S, R);
-        if (int r = launch_check(ctx, "k_window_commit")) return r;
     }
     return FAEDKV_OK;
 }

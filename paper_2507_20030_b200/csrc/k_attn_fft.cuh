@@ -344,7 +344,7 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
                const float2 *__restrict__ Zf, const float *__restrict__ colsum, const int32_t *__restrict__ bins,
                float *__restrict__ partial, unsigned int *__restrict__ tickets, TQ *__restrict__ out,
                int M, int H, int HQ, fft::Geometry g, int bins_per_slice, float inv_P, FoldSrc fold,
-               const float *__restrict__ o_win, int bump) {
+               const float *__restrict__ o_win, int bump, WindowArgs commit) {
     using namespace fft;
     // the weights of a chunk and the final cross-warp reduction share one buffer
     constexpr size_t kWgtBytes = (size_t)kOutChunk * GQ * sizeof(float2) + (APPEND ? kOutChunk * sizeof(float2) : 0);
@@ -466,14 +466,31 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
             store1(out + (size_t)(gcol + q) * kHeadDim + c, s / colsum[gcol + q]);
         }
         if (APPEND && bump) {
-            // every CTA of this sequence has read t_len before taking its ticket; the last CTA of the
-            // sequence's last kv head advances the counter once all H heads are through
+            // every CTA of this sequence has read t_len (and the token it folds) before taking its ticket; the
+            // last CTA of the sequence's last kv head, once all H heads are through, lets the new token take
+            // its ring slot (windowed step) and advances the counter
+            __shared__ unsigned int seq_last;
             if (threadIdx.x == 0) {
                 const unsigned int done = atomicAdd(&tickets[gridDim.y + b], 1u);
-                if (done == (unsigned int)H - 1u) {
-                    tickets[gridDim.y + b] = 0u;
-                    t_len[b] += 1;
+                seq_last = done == (unsigned int)H - 1u ? 1u : 0u;
+                if (seq_last) tickets[gridDim.y + b] = 0u;
+            }
+            __syncthreads();
+            if (seq_last) {
+                const int tt = t_len[b];
+                if (commit.R > 0) {
+                    const int W = commit.S + commit.R, slot = commit.S + (tt - commit.S) % commit.R;
+                    TQ *wK = static_cast<TQ *>(const_cast<void *>(commit.winK)), *wV = static_cast<TQ *>(const_cast<void *>(commit.winV));
+                    const TQ *kn = static_cast<const TQ *>(commit.k_new), *vn = static_cast<const TQ *>(commit.v_new);
+                    for (int e = threadIdx.x; e < H * kHeadDim; e += blockDim.x) {
+                        const size_t unit = (size_t)b * H + e / kHeadDim;
+                        const int c = e % kHeadDim;
+                        wK[(unit * W + slot) * kHeadDim + c] = kn[unit * kHeadDim + c];
+                        wV[(unit * W + slot) * kHeadDim + c] = vn[unit * kHeadDim + c];
+                    }
                 }
+                __syncthreads();
+                if (threadIdx.x == 0) t_len[b] = tt + 1;
             }
         }
     }

@@ -48,82 +48,96 @@ __global__ void k_window_fill(const T *__restrict__ K, const T *__restrict__ V, 
 // unnormalised form as a tile of the transformed segment: per column the maximum score m, the sum of
 // exp(s - m), and o_w[col][c] = sum_w exp(s_w - m) v_w[c].  The slot of the step's new token still holds
 // the token that leaves the window, so k_new / v_new stand in for that row.
-// grid = units; block = 256; dynamic smem = GQ * (S + R) floats.
+// The host runs it on a second stream beside the first two FFT kernels, which leave the memory system idle:
+// beside a bandwidth-saturating pass its dependent loads would each cost many microseconds.
+// grid = (units, GQ): one CTA per query head; block = 256; dynamic smem = (S + R) floats.
+struct WindowArgs {
+    const void *winK, *winV, *k_new, *v_new;   // storage type of the context
+    int S, R;
+    float scale;
+    float *m_w, *s_w, *o_w;                    // statistics row of the window, [Gp] each; output [Gp][128]
+};
+
 template <typename TQ, int GQ>
 __global__ void __launch_bounds__(256)
-k_attn_window(const TQ *__restrict__ q, const TQ *__restrict__ winK, const TQ *__restrict__ winV,
-              const TQ *__restrict__ k_new, const TQ *__restrict__ v_new, const int32_t *__restrict__ t_len, int H,
-              int S, int R, float scale, float *__restrict__ m_w, float *__restrict__ s_w, float *__restrict__ o_w) {
-    extern __shared__ float sc[];                     // [GQ][W]
-
-    const int W = S + R;
+k_attn_window(const TQ *__restrict__ q, WindowArgs wa, const int32_t *__restrict__ t_len, int H) {
+    extern __shared__ float sc[];                     // [W] scores, then exp(s - m)
+    __shared__ float part[kHeadDim];
+    const TQ *winK = static_cast<const TQ *>(wa.winK), *winV = static_cast<const TQ *>(wa.winV);
+    const TQ *k_new = static_cast<const TQ *>(wa.k_new), *v_new = static_cast<const TQ *>(wa.v_new);
+    const int S = wa.S, R = wa.R, W = S + R;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bh = blockIdx.x, b = bh / H;
+    const int bh = blockIdx.x, b = bh / H, col = bh * GQ + (int)blockIdx.y;     // one query head per CTA
     const int t = t_len[b];
     const int slot_new = R > 0 ? S + (t - S) % R : -1;
-    const int col0 = bh * GQ;
-    float4 qv[GQ];
+    const float4 qv = load4(q + (size_t)col * kHeadDim + lane * 4);
+    // scores: a warp takes rows w = warp + 8u, all loads of a batch of 8 issued before any is used
+    for (int w0 = warp; w0 < W; w0 += 64) {
+        float4 kv[8];
 #pragma unroll
-    for (int g = 0; g < GQ; ++g) qv[g] = load4(q + (size_t)(col0 + g) * kHeadDim + lane * 4);
-    for (int w = warp; w < W; w += 8) {
-        const TQ *krow = (w == slot_new) ? k_new + (size_t)bh * kHeadDim : winK + ((size_t)bh * W + w) * kHeadDim;
-        const float4 kv = load4(krow + lane * 4);
+        for (int u = 0; u < 8; ++u) {
+            const int w = w0 + 8 * u;
+            kv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (w < W) {
+                const TQ *krow = (w == slot_new) ? k_new + (size_t)bh * kHeadDim : winK + ((size_t)bh * W + w) * kHeadDim;
+                kv[u] = load4(krow + lane * 4);
+            }
+        }
+        float d[8];
 #pragma unroll
-        for (int g = 0; g < GQ; ++g) {
-            float d = kv.x * qv[g].x + kv.y * qv[g].y + kv.z * qv[g].z + kv.w * qv[g].w;
+        for (int u = 0; u < 8; ++u) d[u] = kv[u].x * qv.x + kv[u].y * qv.y + kv[u].z * qv.z + kv[u].w * qv.w;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-            if (lane == 0) sc[g * W + w] = d * scale;
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int u = 0; u < 8; ++u) d[u] += __shfl_xor_sync(0xffffffffu, d[u], o);     // 8 independent chains
+        if (lane < 8 && w0 + 8 * lane < W) {
+            float v = d[0];
+#pragma unroll
+            for (int u = 1; u < 8; ++u) v = lane == u ? d[u] : v;
+            sc[w0 + 8 * lane] = v * wa.scale;
         }
     }
     __syncthreads();
-    if (warp < GQ) {
+    if (warp == 0) {
         float m = -INFINITY;
-        for (int w = lane; w < W; w += 32) m = fmaxf(m, sc[warp * W + w]);
+        for (int w = lane; w < W; w += 32) m = fmaxf(m, sc[w]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         float sum = 0.f;
         for (int w = lane; w < W; w += 32) {
-            const float p = __expf(sc[warp * W + w] - m);
-            sc[warp * W + w] = p;
+            const float p = __expf(sc[w] - m);
+            sc[w] = p;
             sum += p;
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
         if (lane == 0) {
-            m_w[col0 + warp] = m;
-            s_w[col0 + warp] = sum;
+            wa.m_w[col] = m;
+            wa.s_w[col] = sum;
         }
     }
     __syncthreads();
-    const int c = threadIdx.x & (kHeadDim - 1);
-    for (int g = threadIdx.x >> 7; g < GQ; g += 2) {
-        float acc = 0.f;
-        for (int w = 0; w < W; ++w) {
-            const TQ *vrow = (w == slot_new) ? v_new + (size_t)bh * kHeadDim : winV + ((size_t)bh * W + w) * kHeadDim;
-            acc = fmaf(sc[g * W + w], load1(vrow + c), acc);
+    // output: thread (channel c, half) sums the rows of its parity, 8 loads in flight; halves meet in shared memory
+    const int c = threadIdx.x & (kHeadDim - 1), half = threadIdx.x >> 7;
+    float acc = 0.f;
+    for (int w0 = half; w0 < W; w0 += 16) {
+        float vv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int w = w0 + 2 * u;
+            vv[u] = 0.f;
+            if (w < W) {
+                const TQ *vrow = (w == slot_new) ? v_new + (size_t)bh * kHeadDim : winV + ((size_t)bh * W + w) * kHeadDim;
+                vv[u] = load1(vrow + c);
+            }
         }
-        o_w[(size_t)(col0 + g) * kHeadDim + c] = acc;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (w0 + 2 * u < W) acc = fmaf(sc[w0 + 2 * u], vv[u], acc);
     }
-}
-
-// End of a windowed step: the new token takes its ring slot (R > 0) and the token counters advance.
-// grid = batch; block = 128.
-template <typename T>
-__global__ void k_window_commit(const T *__restrict__ k_new, const T *__restrict__ v_new, T *__restrict__ winK,
-                                T *__restrict__ winV, int32_t *__restrict__ t_len, int H, int S, int R) {
-    const int b = blockIdx.x, c = threadIdx.x;
-    const int t = t_len[b];
-    if (R > 0) {
-        const int slot = S + (t - S) % R;
-        for (int h = 0; h < H; ++h) {
-            const size_t unit = (size_t)b * H + h;
-            winK[(unit * (S + R) + slot) * kHeadDim + c] = k_new[unit * kHeadDim + c];
-            winV[(unit * (S + R) + slot) * kHeadDim + c] = v_new[unit * kHeadDim + c];
-        }
-    }
+    if (half == 1) part[c] = acc;
     __syncthreads();
-    if (c == 0) t_len[b] = t + 1;
+    if (half == 0) wa.o_w[(size_t)col * kHeadDim + c] = acc + part[c];
 }
 
 }  // namespace faedkv
