@@ -226,58 +226,73 @@ def running_mean_step(Sre, Sim, P, bins, t, xnew):
 # Sink and recent window (Sec. 4.2): the paper's own decode workflow for ONE (sequence, kv head) unit,
 # written as a composition of the primitives above -- no new arithmetic.
 class WindowedUnit:
-    """State of one unit: the first S tokens (sink) and the last R tokens (recent) in the time domain,
-    the tokens between them as retained DFT coefficients of the segment that starts at token S."""
+    """State of one unit: the first S tokens (sink) and the most recent tokens in the time domain, the
+    tokens between them as retained DFT coefficients of the segment that starts at token S.
 
-    def __init__(self, P: int, bins: np.ndarray, S: int, R: int):
+    defer = 1 is the paper's step (Eq. 12): every step the token that leaves the R-token recent window is
+    folded into the coefficients.  defer = D > 1 is the block form of the same update: tokens wait in the
+    time domain until R + D of them are unfolded, then the D oldest are folded in one go, oldest first.
+    Whenever (t - S - R) is a multiple of D the two forms hold the same state; in between the block form
+    attends over up to D - 1 more exact tokens."""
+
+    def __init__(self, P: int, bins: np.ndarray, S: int, R: int, defer: int = 1):
         self.P, self.bins, self.S, self.R = int(P), np.ascontiguousarray(bins, dtype=np.int32), int(S), int(R)
+        self.D = int(defer)
+        assert self.D >= 1
         self.t = 0
+        self.folded = 0                              # tokens in the transformed segment
         self.sinkK = self.sinkV = None
-        self.recentK, self.recentV = [], []          # oldest first
+        self.recentK, self.recentV = [], []          # unfolded tokens after the sink, oldest first
         self.CK = self.CV = None                     # (re, im) pairs of [M, d]
 
     def prefill(self, K: np.ndarray, V: np.ndarray) -> None:
-        """Eq. 10: transform K[S : T-R], V[S : T-R]; keep the first S and last R rows as they are."""
+        """Eq. 10: transform K[S : S + folded], V[S : S + folded]; keep the first S rows and the rows after
+        the transformed segment as they are.  folded = T - S - R rounded down to a multiple of defer."""
         K, V = _f64arr(K), _f64arr(V)
         T, d = K.shape
         S, R = self.S, self.R
         assert T >= S + R
+        self.folded = (T - S - R) // self.D * self.D
+        first = S + self.folded                      # first unfolded token
         self.sinkK, self.sinkV = K[:S].copy(), V[:S].copy()
-        self.recentK = [K[n].copy() for n in range(T - R, T)]
-        self.recentV = [V[n].copy() for n in range(T - R, T)]
+        self.recentK = [K[n].copy() for n in range(first, T)]
+        self.recentV = [V[n].copy() for n in range(first, T)]
         M = self.bins.shape[0]
-        if T - S - R > 0:
-            self.CK = [np.ascontiguousarray(a) for a in compress(K[S:T - R], self.P, self.bins)]
-            self.CV = [np.ascontiguousarray(a) for a in compress(V[S:T - R], self.P, self.bins)]
+        if self.folded > 0:
+            self.CK = [np.ascontiguousarray(a) for a in compress(K[S:first], self.P, self.bins)]
+            self.CV = [np.ascontiguousarray(a) for a in compress(V[S:first], self.P, self.bins)]
         else:
             self.CK = [np.zeros((M, d)), np.zeros((M, d))]
             self.CV = [np.zeros((M, d)), np.zeros((M, d))]
         self.t = T
 
     def step(self, k_new: np.ndarray, v_new: np.ndarray) -> None:
-        """Eq. 12: the token leaving the recent window is folded at the next position of the transformed
-        segment; the new token enters the window.  With R = 0 the new token itself is folded."""
+        """Eq. 12: the new token enters the window; once R + defer tokens are unfolded the oldest `defer` of
+        them are folded at the next positions of the transformed segment (defer = 1: the one token leaving
+        the recent window; with R = 0 the new token itself)."""
         k_new, v_new = _f64arr(k_new), _f64arr(v_new)
-        pos = self.t - self.S - self.R                # tokens already in the transformed segment
         self.recentK.append(k_new.copy())
         self.recentV.append(v_new.copy())
-        k_old, v_old = self.recentK.pop(0), self.recentV.pop(0)
-        append(self.CK[0], self.CK[1], self.P, self.bins, pos, k_old)
-        append(self.CV[0], self.CV[1], self.P, self.bins, pos, v_old)
         self.t += 1
+        if len(self.recentK) >= self.R + self.D:
+            for _ in range(self.D):
+                k_old, v_old = self.recentK.pop(0), self.recentV.pop(0)
+                append(self.CK[0], self.CK[1], self.P, self.bins, self.folded, k_old)
+                append(self.CV[0], self.CV[1], self.P, self.bins, self.folded, v_old)
+                self.folded += 1
 
     def attention(self, q: np.ndarray, scale: float | None = None) -> np.ndarray:
-        """Eq. 13 then Eq. 3: one softmax over [sink | reconstructed segment | recent]."""
+        """Eq. 13 then Eq. 3: one softmax over [sink | reconstructed segment | unfolded recent tokens]."""
         q = _f64arr(q)
         d = q.shape[1]
         if scale is None:
             scale = 1.0 / np.sqrt(d)
-        L = min(self.t - self.S - self.R, self.P)
+        L = min(self.folded, self.P)
         parts_k, parts_v = [self.sinkK], [self.sinkV]
         if L > 0:
             parts_k.append(reconstruct(self.CK[0], self.CK[1], self.P, self.bins, L))
             parts_v.append(reconstruct(self.CV[0], self.CV[1], self.P, self.bins, L))
-        if self.R > 0:
+        if self.recentK:
             parts_k.append(np.stack(self.recentK))
             parts_v.append(np.stack(self.recentV))
         Kt = np.concatenate([p for p in parts_k if p.shape[0] > 0], axis=0)

@@ -465,6 +465,65 @@ def test_windowed_folds_the_token_that_leaves_the_window(oracle):
     assert np.array_equal(np.stack(u.recentV), V[t - R:t]) and np.array_equal(u.sinkK, K[:S])
 
 
+@pytest.mark.parametrize("S,R,D", [(3, 5, 4), (0, 4, 3), (2, 0, 5), (0, 0, 2)])
+def test_deferred_all_bins_is_full_attention(oracle, S, R, D):
+    """Block-deferred fold, every bin retained, sequence shorter than the grid: whatever is folded and
+    whatever still waits in the time domain, attention equals textbook attention over all tokens (numpy) at
+    every step, across several block folds."""
+    P, T, d, G, steps = 64, 27, 8, 2, 14
+    rng = np.random.default_rng(100 + S * 10 + R + D)
+    K, V = rng.standard_normal((T + steps, d)), rng.standard_normal((T + steps, d))
+    bins = oracle.plan(P, np.ones(P // 2 + 1, dtype=np.uint8))
+    u = oracle.WindowedUnit(P, bins, S, R, defer=D)
+    u.prefill(K[:T], V[:T])
+    folds = 0
+    for s in range(steps + 1):
+        q = rng.standard_normal((G, d))
+        got = u.attention(q, 0.3)
+        want = _numpy_attention(q, K[:T + s], V[:T + s], 0.3)
+        assert np.abs(got - want).max() < 1e-11, (s, np.abs(got - want).max())
+        assert u.folded % D == 0 and R <= len(u.recentK) < R + D and u.folded + len(u.recentK) + S == u.t
+        if s < steps:
+            before = u.folded
+            u.step(K[T + s], V[T + s])
+            folds += u.folded != before
+    assert folds >= 2
+
+
+def test_deferred_meets_the_per_step_fold_at_block_boundaries(oracle):
+    """Pruned bins: whenever (t - S - R) is a multiple of D the block form holds the state of the
+    per-step form (same coefficients, same window), and the coefficients are the DFT of tokens
+    [S, S + folded) (Eq. 10); in between it has folded fewer tokens and holds more of them exactly."""
+    P, T, d, S, R, D, steps = 32, 19, 4, 2, 3, 4, 11
+    rng = np.random.default_rng(21)
+    K, V = rng.standard_normal((T + steps, d)), rng.standard_normal((T + steps, d))
+    mask = np.zeros(P // 2 + 1, dtype=np.uint8)
+    mask[[0, 2, 7, 16]] = 1
+    bins = oracle.plan(P, mask)
+    a, b = oracle.WindowedUnit(P, bins, S, R), oracle.WindowedUnit(P, bins, S, R, defer=D)
+    a.prefill(K[:T], V[:T])
+    b.prefill(K[:T], V[:T])
+    hits = 0
+    for s in range(steps + 1):
+        t = T + s
+        assert b.folded == (t - S - R) // D * D
+        re, im = oracle.compress(V[S:S + b.folded], P, bins) if b.folded else (0 * b.CV[0], 0 * b.CV[1])
+        assert np.abs(b.CV[0] - re).max() < 1e-11 and np.abs(b.CV[1] - im).max() < 1e-11
+        assert np.array_equal(np.stack(b.recentK), K[S + b.folded:t])
+        if (t - S - R) % D == 0:
+            hits += 1
+            assert np.abs(a.CK[0] - b.CK[0]).max() < 1e-11 and np.abs(a.CK[1] - b.CK[1]).max() < 1e-11
+            assert np.array_equal(np.stack(a.recentV), np.stack(b.recentV))
+            q = rng.standard_normal((2, d))
+            assert np.abs(a.attention(q) - b.attention(q)).max() < 1e-12
+        else:
+            assert b.folded < a.folded and len(b.recentK) > R
+        if s < steps:
+            a.step(K[t], V[t])
+            b.step(K[t], V[t])
+    assert hits >= 3
+
+
 # ----------------------------------------------------------------------------- ablation and selection
 def test_chunk_ranges_partition_the_grid(oracle):
     for P, C in [(64, 22), (100, 7), (2048, 22), (22, 22)]:
