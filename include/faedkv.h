@@ -96,6 +96,8 @@ typedef struct {
                           uses 10).  Only the *_windowed calls look at n_sink / n_recent */
     int n_recent;      /* R >= 0: most recent tokens kept in the time domain (the paper
                           uses 50); n_sink + n_recent <= 1024                        */
+    int n_defer;       /* D: 0 or 1 = the paper's step, one token folded per step (Eq. 12);
+                          2 .. 128 = block-deferred fold, see the window section       */
 } faedkv_config;
 
 /* Create a context on the CURRENT CUDA device.  Allocates the scratch area
@@ -192,7 +194,16 @@ int faedkv_append_decode_attn(faedkv_ctx *ctx, int layer, const void *k_new, con
  *   [batch][n_kv_heads][S + R][head_dim]:  rows [0, S) the sink tokens, rows [S, S + R) a ring in
  *   which token n >= S occupies slot (n - S) mod R while it is among the last R tokens.
  * t_len counts ALL tokens of a sequence; the transformed segment holds t_len - S - R of them, at
- * positions 0, 1, ... (token n sits at position n - S), wrapping modulo P like everywhere else. */
+ * positions 0, 1, ... (token n sits at position n - S), wrapping modulo P like everywhere else.
+ *
+ * Block-deferred fold (n_defer = D >= 2).  Eq. 12 costs a read and a write of every coefficient per
+ * step.  Because the update is linear, tokens may instead wait in the time domain and be folded D at
+ * a time: the ring then has R + D slots (rows [S, S + R + D); token n in slot (n - S) mod (R + D)),
+ * the transformed segment holds  folded(t) = D * floor((t - S - R) / D)  tokens (0 while t < S + R),
+ * and a step whose token brings t - S - R to a multiple of D folds the D oldest waiting tokens,
+ * oldest first, with exactly the arithmetic of D single-token updates.  Whenever t - S - R is a
+ * multiple of D the state equals that of the per-step form; in between, up to D - 1 more tokens are
+ * attended exactly instead of through their retained bins.  Every other step only READS the planes. */
 
 /* Bytes of ONE window tensor (K or V) at this batch. */
 size_t faedkv_window_bytes(const faedkv_ctx *ctx, int batch);
@@ -200,6 +211,7 @@ size_t faedkv_window_bytes(const faedkv_ctx *ctx, int batch);
 /* Prefill (Eq. 10): tokens [0, S) are copied to the sink rows, tokens [T - R, T) to their ring
  * slots, and the tokens between them are transformed into coefK, coefV as in
  * faedkv_compress_prefill (planes are zero when there is none).  SETS t_len[b] = T.
+ * With n_defer = D >= 2 the transformed tokens are [S, S + folded(T)) and the ring takes the rest.
  * T >= S + R is required (FAEDKV_ERR_SHAPE otherwise).  With S = R = 0 this is
  * faedkv_compress_prefill and winK, winV may be NULL. */
 int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch,
@@ -214,6 +226,10 @@ int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const voi
  *                    and the R most recent tokens including the new one -- one softmax, evaluated
  *                    without writing K~, V~ or the scores to memory;
  *   commit           the new token takes the ring slot of the one that left; t_len[b] += 1.
+ * With n_defer = D >= 2: the D oldest waiting tokens are folded if t + 1 - S - R is a multiple of D
+ * (per sequence; ragged batches fold at different steps), attention runs over the sink, the
+ * reconstruction of min(folded(t + 1), P) positions and all waiting tokens including the new one,
+ * then the new token takes its ring slot and t_len[b] += 1.
  * Needs the FFT-shaped decode path (P a power of two in [64, 2^19]); FAEDKV_ERR_UNSUPPORTED
  * otherwise.  winK, winV, coefK, coefV and t_len are updated in place. */
 int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new,

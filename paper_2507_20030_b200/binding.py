@@ -45,7 +45,7 @@ class FaedkvError(RuntimeError):
 class Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "n_layers", "n_kv_heads", "n_q_heads", "head_dim", "n_dft", "max_batch", "kv_dtype",
-        "prefill_mode", "twiddle_terms", "decode_mode", "n_sink", "n_recent")]
+        "prefill_mode", "twiddle_terms", "decode_mode", "n_sink", "n_recent", "n_defer")]
 
 
 _lib = None
@@ -212,12 +212,13 @@ class Context:
     decode_mode: int = DECODE_AUTO
     n_sink: int = 0
     n_recent: int = 0
+    n_defer: int = 0
 
     def __post_init__(self):
         self._lib = load()
         cfg = Config(self.n_layers, self.n_kv_heads, self.n_q_heads, self.head_dim, self.n_dft,
                      self.max_batch, self.kv_dtype, self.prefill_mode, self.twiddle_terms, self.decode_mode,
-                     self.n_sink, self.n_recent)
+                     self.n_sink, self.n_recent, self.n_defer)
         h = _vp()
         rc = self._lib.faedkv_create(ctypes.byref(cfg), ctypes.byref(h))
         if rc != 0:
@@ -319,8 +320,10 @@ class Context:
 
     # -- sink + recent window
     def alloc_window(self, batch: int, device="cuda") -> torch.Tensor:
-        """[batch, n_kv_heads, n_sink + n_recent, head_dim] in the storage type (uninitialised)."""
-        return torch.empty((batch, self.n_kv_heads, self.n_sink + self.n_recent, self.head_dim),
+        """[batch, n_kv_heads, n_sink + ring, head_dim] in the storage type (uninitialised); the ring has
+        n_recent slots, or n_recent + n_defer with the block-deferred fold (n_defer >= 2)."""
+        ring = self.n_recent + (self.n_defer if self.n_defer > 1 else 0)
+        return torch.empty((batch, self.n_kv_heads, self.n_sink + ring, self.head_dim),
                            dtype=self.torch_dtype, device=device)
 
     def prefill_windowed(self, layer, K, V, coefK, coefV, winK, winV, t_len, stream=None):

@@ -56,7 +56,7 @@ struct FftScratch {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     unsigned int *tickets = nullptr;      // [max_batch * H + max_batch], zero between calls
     int max_M = 0;
-    unsigned int attr_mask[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
+    unsigned int attr_mask[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
 };
 
 }  // namespace
@@ -202,7 +202,7 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             CUDA_TRY(ctx, cudaMalloc(&f.mloc, (size_t)(g.N1 + 1) * g.Gp * sizeof(float)));
             CUDA_TRY(ctx, cudaMalloc(&f.sloc, (size_t)(g.N1 + 1) * g.Gp * sizeof(float)));
             CUDA_TRY(ctx, cudaMalloc(&f.colsum, (size_t)2 * g.Gp * sizeof(float)));
-            if (c.n_sink + c.n_recent > 0) {
+            if (c.n_sink + c.n_recent > 0 || c.n_defer > 1) {
                 CUDA_TRY(ctx, cudaMalloc(&f.o_win, (size_t)g.Gp * kHeadDim * sizeof(float)));
                 CUDA_TRY(ctx, cudaStreamCreateWithFlags(&f.side, cudaStreamNonBlocking));
                 CUDA_TRY(ctx, cudaEventCreateWithFlags(&f.ev_fork, cudaEventDisableTiming));
@@ -571,7 +571,11 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
     FftScratch &f = ctx->fs;
     const bool windowed = winK != nullptr;
     const int S = windowed ? c.n_sink : 0, R = windowed ? c.n_recent : 0;
-    const int n_extra = (windowed && S + R > 0) ? 1 : 0;
+    // block-deferred fold (D > 1, APPEND == false): the caller has folded already; this call attends over the
+    // whole blocks in the planes plus every waiting token, then commits the new token and advances t_len
+    const int D = windowed ? c.n_defer : 1, Rc = win_ring(R, D);
+    const bool counts_new = APPEND || D > 1;
+    const int n_extra = (windowed && (S + R > 0 || D > 1)) ? 1 : 0;
     // the folded token: the call's new token, or with a ring the token that leaves it
     const FoldSrc fold{(windowed && R > 0) ? S + R : 1, S, R};
     const void *foldK = (windowed && R > 0) ? winK : k_new, *foldV = (windowed && R > 0) ? winV : v_new;
@@ -593,11 +597,11 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         // second stream beside the next two kernels (which leave the memory system idle); joined before the
         // kernel that reads the statistics
         const int n_tiles = g.N1 >> lgMT;
-        const WindowArgs wa{winK, winV, k_new, v_new, S, R, scale, f.mloc + (size_t)n_tiles * g.Gp,
+        const WindowArgs wa{winK, winV, k_new, v_new, S, R, D, Rc, scale, f.mloc + (size_t)n_tiles * g.Gp,
                             f.sloc + (size_t)n_tiles * g.Gp, f.o_win};
         CUDA_TRY(ctx, cudaEventRecord(f.ev_fork, st));
         CUDA_TRY(ctx, cudaStreamWaitEvent(f.side, f.ev_fork, 0));
-        k_attn_window<TQ, GQ><<<dim3(batch * H, GQ), 256, (size_t)(S + R) * sizeof(float), f.side>>>(static_cast<const TQ *>(q), wa, t_len, H);
+        k_attn_window<TQ, GQ><<<dim3(batch * H, GQ), 256, (size_t)(S + Rc) * sizeof(float), f.side>>>(static_cast<const TQ *>(q), wa, t_len, H);
         if (int r = launch_check(ctx, "k_attn_window")) return r;
         CUDA_TRY(ctx, cudaEventRecord(f.ev_join, f.side));
     }
@@ -619,7 +623,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         const size_t smem = afft_smem_mid(g.lgN2, lgMT);
 #define CALL(LG)                                                                                         \
         rc = fft_opt_in(ctx, FFT_PICK(k_afft_mid, LG, lgMT), smem, f.attr_mask[1], LG + ((lgMT) == fft::fast_lg_transforms(LG) ? 16 : 0));                                  \
-        if (rc == 0) launch_pdl(FFT_PICK(k_afft_mid, LG, lgMT), grid, dim3(fft::kThreads), smem, st, g, f.Y, t_len, HQ, (APPEND ? 1 : 0) - S - R, f.mloc, f.sloc, lgMT)
+        if (rc == 0) launch_pdl(FFT_PICK(k_afft_mid, LG, lgMT), grid, dim3(fft::kThreads), smem, st, g, f.Y, t_len, HQ, (counts_new ? 1 : 0) - S - R, D, f.mloc, f.sloc, lgMT)
         FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
 #undef CALL
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
@@ -644,8 +648,8 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         dim3 grid(slices, batch * H);
         launch_pdl(k_attn_out_fft<TQ, GQ, APPEND>, grid, dim3(kAttnWarps * 32), 0, st,
                    coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
-                   static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, 1,
-                   windowed ? WindowArgs{winK, winV, k_new, v_new, S, R, 0.f, nullptr, nullptr, nullptr} : WindowArgs{});
+                   static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, counts_new ? 1 : 0,
+                   windowed ? WindowArgs{winK, winV, k_new, v_new, S, R, D, Rc, 0.f, nullptr, nullptr, nullptr} : WindowArgs{});
         if (int r = launch_check(ctx, "k_attn_out_fft")) return r;
     }
     return FAEDKV_OK;
@@ -831,6 +835,7 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     if (cfg->decode_mode == FAEDKV_DECODE_UMMA && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->decode_mode == FAEDKV_DECODE_FFT && !fft::supported(cfg->n_dft)) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_sink < 0 || cfg->n_recent < 0 || cfg->n_sink + cfg->n_recent > 1024) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->n_defer < 0 || cfg->n_defer > 128) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->head_dim != kHeadDim) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FAEDKV_ERR_UNSUPPORTED;
     const int gq = cfg->n_q_heads / cfg->n_kv_heads;
@@ -1088,7 +1093,7 @@ int faedkv_append_decode_attn(faedkv_ctx *ctx, int layer, const void *k_new, con
 size_t faedkv_window_bytes(const faedkv_ctx *ctx, int batch) {
     if (ctx == nullptr || batch < 1) return 0;
     const size_t elem = ctx->cfg.kv_dtype == FAEDKV_BF16 ? 2 : 4;
-    return (size_t)batch * ctx->cfg.n_kv_heads * (ctx->cfg.n_sink + ctx->cfg.n_recent) * kHeadDim * elem;
+    return (size_t)batch * ctx->cfg.n_kv_heads * (ctx->cfg.n_sink + win_ring(ctx->cfg.n_recent, ctx->cfg.n_defer)) * kHeadDim * elem;
 }
 
 int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch, int T, float *coefK,
@@ -1097,9 +1102,9 @@ int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const voi
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
     const faedkv_config &c = ctx->cfg;
-    const int S = c.n_sink, R = c.n_recent;
+    const int S = c.n_sink, R = c.n_recent, D = c.n_defer, Rc = win_ring(R, D);
     if (K == nullptr || V == nullptr || coefK == nullptr || coefV == nullptr || t_len == nullptr ||
-        (S + R > 0 && (winK == nullptr || winV == nullptr)))
+        (S + Rc > 0 && (winK == nullptr || winV == nullptr)))
         return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_prefill_windowed");
     if (T < S + R || T < 1)
         return fail(ctx, FAEDKV_ERR_SHAPE, "T = %d must cover the sink and recent windows (%d + %d)", T, S, R);
@@ -1107,9 +1112,9 @@ int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const voi
     if (int r = check_tlen(ctx, t_len)) return r;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t elem = c.kv_dtype == FAEDKV_BF16 ? 2 : 4;
-    const int mid = T - S - R;
+    const int mid = win_folded(T, S, R, D);
     if (mid > 0) {
-        // rows [S, T - R) of every unit, at positions 0 .. mid - 1 of the transformed segment (Eq. 10)
+        // rows [S, S + mid) of every unit, at positions 0 .. mid - 1 of the transformed segment (Eq. 10)
         const char *Km = static_cast<const char *>(K) + (size_t)S * kHeadDim * elem;
         const char *Vm = static_cast<const char *>(V) + (size_t)S * kHeadDim * elem;
         if (int r = prefill_core(ctx, *p, Km, Vm, batch, mid, T, coefK, coefV, st)) return r;
@@ -1118,14 +1123,14 @@ int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const voi
         CUDA_TRY(ctx, cudaMemsetAsync(coefK, 0, bytes, st));
         CUDA_TRY(ctx, cudaMemsetAsync(coefV, 0, bytes, st));
     }
-    if (S + R > 0) {
-        dim3 grid(S + R, batch * c.n_kv_heads);
+    if (T - mid > 0) {
+        dim3 grid(T - mid, batch * c.n_kv_heads);      // sink rows + the tokens that stay in the time domain
         if (c.kv_dtype == FAEDKV_BF16)
             k_window_fill<__nv_bfloat16><<<grid, kHeadDim, 0, st>>>(static_cast<const __nv_bfloat16 *>(K), static_cast<const __nv_bfloat16 *>(V),
-                                                                   static_cast<__nv_bfloat16 *>(winK), static_cast<__nv_bfloat16 *>(winV), T, S, R);
+                                                                   static_cast<__nv_bfloat16 *>(winK), static_cast<__nv_bfloat16 *>(winV), T, S, Rc, mid);
         else
             k_window_fill<float><<<grid, kHeadDim, 0, st>>>(static_cast<const float *>(K), static_cast<const float *>(V),
-                                                           static_cast<float *>(winK), static_cast<float *>(winV), T, S, R);
+                                                           static_cast<float *>(winK), static_cast<float *>(winV), T, S, Rc, mid);
         if (int r = launch_check(ctx, "k_window_fill")) return r;
     }
     k_set_tlen<<<(batch + 127) / 128, 128, 0, st>>>(t_len, batch, T);
@@ -1148,7 +1153,27 @@ int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const vo
         return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "the windowed step needs the FFT-shaped decode path (P a power of two in [64, 2^19])");
     if (scale == 0.0f) scale = 1.0f / sqrtf((float)ctx->cfg.head_dim);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (ctx->cfg.kv_dtype == FAEDKV_BF16)
+    const faedkv_config &c = ctx->cfg;
+    if (c.n_defer > 1) {
+        // block-deferred fold: fold the sequences that reach a block boundary (the others' CTAs return at
+        // once), then attend without touching the planes again
+        const int D = c.n_defer;
+        const WindowArgs wa{winK, winV, k_new, v_new, c.n_sink, c.n_recent, D, win_ring(c.n_recent, D), 0.f, nullptr, nullptr, nullptr};
+        const dim3 grid((p->M + kFoldWarps * kFoldBins - 1) / (kFoldWarps * kFoldBins), batch * c.n_kv_heads, 2);
+        const size_t smem = block_fold_smem(D);
+        if (c.kv_dtype == FAEDKV_BF16) {
+            if (int r = fft_opt_in(ctx, k_block_fold<__nv_bfloat16>, smem, ctx->fs.attr_mask[9], 0)) return r;
+            k_block_fold<__nv_bfloat16><<<grid, kFoldWarps * 32, smem, st>>>(coefK, coefV, t_len, p->d_bins, wa, p->M, c.n_kv_heads, (uint32_t)c.n_dft);
+        } else {
+            if (int r = fft_opt_in(ctx, k_block_fold<float>, smem, ctx->fs.attr_mask[9], 1)) return r;
+            k_block_fold<float><<<grid, kFoldWarps * 32, smem, st>>>(coefK, coefV, t_len, p->d_bins, wa, p->M, c.n_kv_heads, (uint32_t)c.n_dft);
+        }
+        if (int r = launch_check(ctx, "k_block_fold")) return r;
+        if (c.kv_dtype == FAEDKV_BF16)
+            return dispatch_attn_fft<__nv_bfloat16, false>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+        return dispatch_attn_fft<float, false>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+    }
+    if (c.kv_dtype == FAEDKV_BF16)
         return dispatch_attn_fft<__nv_bfloat16, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
     return dispatch_attn_fft<float, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
 }

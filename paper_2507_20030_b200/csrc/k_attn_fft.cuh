@@ -145,7 +145,7 @@ k_afft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float2 *__
 // grid = (N1 / MT, Gp / 16); block = 256; dynamic smem = afft_smem_mid(lgN2, lgMT).
 template <int LG, int LGT>
 __global__ void __launch_bounds__(fft::kThreads)
-k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ t_len, int HQ, int t_add,
+k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ t_len, int HQ, int t_add, int t_quant,
            float *__restrict__ mloc, float *__restrict__ sloc, int lgMT_rt) {
     const int lgMT = LGT >= 0 ? LGT : lgMT_rt;   // compile-time in the fast instances
     using namespace fft;
@@ -170,7 +170,8 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
         const int col = g0 + threadIdx.x;
         int live = 0;
         if (col < g.G) {
-            const long long t = (long long)t_len[col / HQ] + t_add;
+            long long t = (long long)t_len[col / HQ] + t_add;
+            if (t_quant > 1 && t > 0) t = t / t_quant * t_quant;      // block-deferred fold: whole blocks only
             live = t < (long long)g.P ? (int)t : (int)g.P;
         }
         live_s[threadIdx.x] = live;
@@ -465,7 +466,7 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
             if (o_win != nullptr) s = fmaf(o_win[(size_t)(gcol + q) * kHeadDim + c], colsum[g.Gp + gcol + q], s);
             store1(out + (size_t)(gcol + q) * kHeadDim + c, s / colsum[gcol + q]);
         }
-        if (APPEND && bump) {
+        if (bump) {
             // every CTA of this sequence has read t_len (and the token it folds) before taking its ticket; the
             // last CTA of the sequence's last kv head, once all H heads are through, lets the new token take
             // its ring slot (windowed step) and advances the counter
@@ -478,8 +479,8 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
             __syncthreads();
             if (seq_last) {
                 const int tt = t_len[b];
-                if (commit.R > 0) {
-                    const int W = commit.S + commit.R, slot = commit.S + (tt - commit.S) % commit.R;
+                if (commit.Rc > 0) {
+                    const int W = commit.S + commit.Rc, slot = commit.S + (tt - commit.S) % commit.Rc;
                     TQ *wK = static_cast<TQ *>(const_cast<void *>(commit.winK)), *wV = static_cast<TQ *>(const_cast<void *>(commit.winV));
                     const TQ *kn = static_cast<const TQ *>(commit.k_new), *vn = static_cast<const TQ *>(commit.v_new);
                     for (int e = threadIdx.x; e < H * kHeadDim; e += blockDim.x) {

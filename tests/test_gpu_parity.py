@@ -576,6 +576,129 @@ def test_windowed_step_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, S, R
     ctx.close()
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("P,Ts,M,H,HQ,S,R,D,steps", [
+    (256, (200, 187), 40, 2, 8, 10, 50, 16, 40),   # the paper's window; a ragged batch folds at different steps
+    (128, (64,), 65, 3, 3, 4, 7, 5, 23),           # every bin retained; MHA; several block folds
+    (512, (530, 529), 33, 1, 2, 0, 16, 8, 20),     # no sink; the transformed segment is longer than P (wraps)
+    (64, (31,), 9, 2, 4, 6, 0, 4, 10),             # no recent window: a block can end with the step's own token
+    (64, (20, 21), 9, 1, 1, 0, 0, 2, 7),           # no window at all: nothing waits at a block boundary
+    (1024, (60,), 24, 2, 4, 10, 50, 128, 140),     # T = S + R: the planes start empty; the largest block
+])
+def test_deferred_step_matches_oracle(fk, oracle, dtype, P, Ts, M, H, HQ, S, R, D, steps):
+    """Block-deferred fold: prefill (one call per sequence, so that the batch is ragged), then decode steps
+    over the whole batch: attention outputs at every step, final planes, ring contents and counters against
+    the oracle's WindowedUnit(defer=D), unit by unit."""
+    from paper_2507_20030_b200 import synth
+    B, GQ = len(Ts), HQ // H
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                     prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R, n_defer=D)
+    mask = _random_mask(P, M, 17 * P + Ts[0])
+    mask[0] = 1
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    Rc = R + D
+    assert ctx._lib.faedkv_window_bytes(ctx._h, B) == B * H * (S + Rc) * 128 * (4 if dtype == torch.float32 else 2)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    cK.fill_(float("nan")); cV.fill_(float("nan"))
+    wK, wV = ctx.alloc_window(B), ctx.alloc_window(B)
+    assert wK.shape == (B, H, S + Rc, 128)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    units = {}
+    for b, T in enumerate(Ts):
+        K, V = _make(61 + P + T + b, 1, H, T, dtype)
+        V = (V * 0.25).to(dtype)
+        for h in range(H):
+            u = units[(b, h)] = oracle.WindowedUnit(P, bins, S, R, defer=D)
+            u.prefill(to_np64(K[0, h]), to_np64(V[0, h]))
+        ctx.prefill_windowed(0, K.cuda(), V.cuda(), cK[b:b + 1], cV[b:b + 1], wK[b:b + 1], wV[b:b + 1], t_len[b:b + 1])
+    assert t_len.tolist() == list(Ts)
+    out = torch.empty((B, HQ, 128), dtype=dtype, device="cuda")
+    folds = 0
+    for s in range(steps):
+        k, v = synth.make_token(79, s, B, H, 128, pos=Ts[0] + s, dtype=dtype)
+        v = (v * 0.25).to(dtype)
+        q = synth.make_q(79, s, B, HQ, 128, dtype=dtype)
+        ctx.step_windowed(0, k.cuda(), v.cuda(), q.cuda(), cK, cV, wK, wV, t_len, out)
+        torch.cuda.synchronize()
+        got = to_np64(out)
+        for (b, h), u in units.items():
+            before = u.folded
+            u.step(to_np64(k[b, h]), to_np64(v[b, h]))
+            folds += u.folded != before
+            want = u.attention(to_np64(q[b, h * GQ:(h + 1) * GQ]))
+            err = np.abs(got[b, h * GQ:(h + 1) * GQ] - want).max()
+            assert err <= ATTN_MAX_ABS, (s, b, h, err)
+    assert folds >= B * H                      # every unit went through at least one block fold
+    assert t_len.tolist() == [T + steps for T in Ts] and ctx.device_status() == 0
+    gK, gV, gwK, gwV = to_np64(cK), to_np64(cV), to_np64(wK), to_np64(wV)
+    for (b, h), u in units.items():
+        assert rel_l2(gK[b, h], np.stack(u.CK)) <= REL_L2_F32 and rel_l2(gV[b, h], np.stack(u.CV)) <= REL_L2_F32
+        assert np.array_equal(gwK[b, h, :S], u.sinkK)
+        t = Ts[b] + steps
+        first = S + u.folded
+        assert u.folded == max(0, (t - S - R) // D * D) and len(u.recentK) == t - first
+        for j, n in enumerate(range(first, t)):   # ring slot of token n is (n - S) mod (R + D)
+            assert np.array_equal(gwK[b, h, S + (n - S) % Rc], u.recentK[j]), (b, h, n)
+            assert np.array_equal(gwV[b, h, S + (n - S) % Rc], u.recentV[j]), (b, h, n)
+    ctx.close()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("S,R,D", [(0, 0, 4), (3, 6, 5), (10, 50, 32)])
+def test_block_fold_is_bit_identical_to_single_token_updates(fk, dtype, S, R, D):
+    """At every block boundary the planes of the block-deferred form equal, bit for bit, those of the
+    per-step form fed the same tokens (the block fold performs the same FMAs in the same order); with no
+    window at all the per-step form is faedkv_append."""
+    from paper_2507_20030_b200 import synth
+    P, M, B, H, HQ = 256, 48, 2, 2, 4
+    T = S + R + 3 * D                              # prefill ends on a block boundary
+    mask = _random_mask(P, M, 5)
+    ctxs = [fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                       prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R, n_defer=d) for d in (1, D)]
+    K, V = _make(3, B, H, T, dtype)
+    st = []
+    for ctx in ctxs:
+        ctx.plan(0, mask)
+        cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+        wK, wV = ctx.alloc_window(B), ctx.alloc_window(B)
+        t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+        ctx.prefill_windowed(0, K.cuda(), V.cuda(), cK, cV, wK, wV, t_len)
+        st.append((cK, cV, wK, wV, t_len))
+    assert torch.equal(st[0][0], st[1][0]) and torch.equal(st[0][1], st[1][1])
+    plain = None
+    if S + R == 0:                                 # third arm: the plain append call
+        pc = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                        prefill_mode=fk.PREFILL_SIMT)
+        pc.plan(0, mask)
+        plain = (pc, st[0][0].clone(), st[0][1].clone(), st[0][4].clone())
+    out = torch.empty((B, HQ, 128), dtype=dtype, device="cuda")
+    checked = 0
+    for s in range(2 * D + 1):
+        k, v = synth.make_token(83, s, B, H, 128, pos=T + s, dtype=dtype)
+        q = synth.make_q(83, s, B, HQ, 128, dtype=dtype)
+        for ctx, (cK, cV, wK, wV, t_len) in zip(ctxs, st):
+            if S + R == 0 and ctx.n_defer <= 1:    # no window tensor at all: the per-step form is the fused call
+                ctx.append_decode_attn(0, k.cuda(), v.cuda(), q.cuda(), cK, cV, t_len, out)
+            else:
+                ctx.step_windowed(0, k.cuda(), v.cuda(), q.cuda(), cK, cV, wK, wV, t_len, out)
+        if plain is not None:
+            plain[0].append(0, k.cuda(), v.cuda(), plain[1], plain[2], plain[3])
+        torch.cuda.synchronize()
+        same = torch.equal(st[0][0], st[1][0]) and torch.equal(st[0][1], st[1][1])
+        if (T + s + 1 - S - R) % D == 0:
+            assert same, s
+            if plain is not None:
+                assert torch.equal(plain[1], st[1][0]) and torch.equal(plain[2], st[1][1]), s
+            checked += 1
+        else:
+            assert not same, s                     # between boundaries the deferred planes lag behind
+    assert checked == 2
+    for ctx in ctxs:
+        assert ctx.device_status() == 0
+        ctx.close()
+
+
 def test_windowed_rejects_short_prefill_and_non_fft_grids(fk):
     ctx = fk.Context(n_layers=1, n_kv_heads=1, n_q_heads=1, n_dft=100, max_batch=1, kv_dtype=fk.F32, n_sink=4, n_recent=8)
     ctx.plan(0, _mask_from_bins(100, [0, 1, 2]))
