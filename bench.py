@@ -275,6 +275,56 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     if graphs:
         res["decode_us_per_layer_step"] = res["append_decode_attn"]["us"]
         res["decode_us_per_layer_step_two_calls"] = res["append"]["us"] + res["decode_attn"]["us"]
+    # the same windowed workflow with the block-deferred fold: 50 tokens folded at once every 50th step, the
+    # other steps only read the planes.  All layers' steps (one CUDA graph, or eager launches) are run 50
+    # times, each run timed; the counters are first set so that the first of the 50 is the one that folds.
+    DEFER, S_, R_ = 50, 10, 50
+    ctx2 = binding.Context(n_layers=NL, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=binding.BF16,
+                           n_sink=S_, n_recent=R_, n_defer=DEFER)
+    for l in range(NL):
+        ctx2.plan(l, binding.mask_mixed(P, M, l, seed))
+    w2K, w2V = synth.make_kv(seed + 9, B, H, S_ + R_ + DEFER, D, pos0=T - 60 - DEFER, dtype=torch.bfloat16, device=dev)
+    fn = lambda: [ctx2.step_windowed(l, k_new, v_new, q, cKs[l], cVs[l], w2K, w2V, tls[l], out) for l in range(NL)]
+    t_now = int(tls[0][0].item())
+    t_fold = S_ + R_ + ((t_now - S_ - R_) // DEFER + 2) * DEFER - 1      # a step from this count folds
+    run = fn
+    if graphs:
+        for tl in tls:
+            tl.fill_(t_fold - 3)
+        graph = torch.cuda.CUDAGraph()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.synchronize()
+        run = graph.replay
+        for _ in range(2):
+            run()
+    else:
+        for tl in tls:
+            tl.fill_(t_fold)
+    torch.cuda.synchronize()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(DEFER + 1)]
+    evs[0].record()
+    for i in range(DEFER):
+        run()
+        evs[i + 1].record()
+    torch.cuda.synchronize()
+    per = [evs[i].elapsed_time(evs[i + 1]) / NL * 1e3 for i in range(DEFER)]
+    us = evs[0].elapsed_time(evs[DEFER]) / DEFER / NL * 1e3
+    nbytes = coef_bytes + 2 * coef_bytes / DEFER
+    gbs = nbytes / (us * 1e-6) / 1e9
+    res["step_windowed_deferred"] = {
+        "us": us, "us_step_without_fold": sorted(per)[len(per) // 2], "us_step_with_fold": per[0], "defer": DEFER,
+        "launch": "one CUDA graph per step of all layers" if graphs else "eager launches",
+        "bytes": nbytes, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"],
+        "what": "mean over 50 consecutive steps, the first of which folds 50 tokens into every layer's planes; "
+                "bytes = planes read once per step + read and written once per 50 steps"}
+    if ctx2.device_status() != 0:
+        raise RuntimeError("a kernel reported a device-side timeout; the numbers are invalid")
+    ctx2.close()
     if ctx.device_status() != 0:
         raise RuntimeError("a kernel reported a device-side timeout; the numbers are invalid")
     ctx.close()

@@ -585,25 +585,25 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
     const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks));
     const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks));
     constexpr int KB = 16 / GQ;
+    if (n_extra) {
+        // the window's scores, statistics (one more "tile" row) and unnormalised output depend on nothing this call
+        // computes: they run on the context's second stream from the top of the call, beside the pass over
+        // C_K, and are joined before the kernel that reads the statistics
+        const int n_tiles = g.N1 >> lgMT;
+        const WindowArgs wa{winK, winV, k_new, v_new, S, R, D, Rc, scale, f.mloc + (size_t)n_tiles * g.Gp,
+                            f.sloc + (size_t)n_tiles * g.Gp, f.o_win};
+        CUDA_TRY(ctx, cudaEventRecord(f.ev_fork, st));
+        CUDA_TRY(ctx, cudaStreamWaitEvent(f.side, f.ev_fork, 0));
+        k_attn_window<TQ, GQ><<<dim3(batch * H, GQ), kWinWarps * 32, 0, f.side>>>(static_cast<const TQ *>(q), wa, t_len, H);
+        if (int r = launch_check(ctx, "k_attn_window")) return r;
+        CUDA_TRY(ctx, cudaEventRecord(f.ev_join, f.side));
+    }
     {
         dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
         k_attn_qs<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(
             static_cast<const TQ *>(q), coefK, static_cast<const TQ *>(foldK), t_len, p.d_bins, f.Qs, M, H, HQ, g.Gp,
             (uint32_t)P, scale / (float)P, fold);
         if (int r = launch_check(ctx, "k_attn_qs")) return r;
-    }
-    if (n_extra) {
-        // the window's scores, statistics (one more "tile" row) and unnormalised output, on the context's
-        // second stream beside the next two kernels (which leave the memory system idle); joined before the
-        // kernel that reads the statistics
-        const int n_tiles = g.N1 >> lgMT;
-        const WindowArgs wa{winK, winV, k_new, v_new, S, R, D, Rc, scale, f.mloc + (size_t)n_tiles * g.Gp,
-                            f.sloc + (size_t)n_tiles * g.Gp, f.o_win};
-        CUDA_TRY(ctx, cudaEventRecord(f.ev_fork, st));
-        CUDA_TRY(ctx, cudaStreamWaitEvent(f.side, f.ev_fork, 0));
-        k_attn_window<TQ, GQ><<<dim3(batch * H, GQ), 256, (size_t)(S + Rc) * sizeof(float), f.side>>>(static_cast<const TQ *>(q), wa, t_len, H);
-        if (int r = launch_check(ctx, "k_attn_window")) return r;
-        CUDA_TRY(ctx, cudaEventRecord(f.ev_join, f.side));
     }
     int rc = FAEDKV_ERR_UNSUPPORTED;
     {
@@ -1159,14 +1159,19 @@ int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const vo
         // once), then attend without touching the planes again
         const int D = c.n_defer;
         const WindowArgs wa{winK, winV, k_new, v_new, c.n_sink, c.n_recent, D, win_ring(c.n_recent, D), 0.f, nullptr, nullptr, nullptr};
-        const dim3 grid((p->M + kFoldWarps * kFoldBins - 1) / (kFoldWarps * kFoldBins), batch * c.n_kv_heads, 2);
+        // work items (sequence, 32 bins, share of the 2H planes); the planes are split until the items fill the SMs
+        const int n_groups = (p->M + kFoldGroup - 1) / kFoldGroup;
+        int splits = 1;
+        while (splits < 2 * c.n_kv_heads && batch * n_groups * splits < 4 * 148) splits *= 2;
+        const int n_items = batch * n_groups * splits;
+        const dim3 grid(n_items < 4 * 148 ? n_items : 4 * 148);
         const size_t smem = block_fold_smem(D);
         if (c.kv_dtype == FAEDKV_BF16) {
             if (int r = fft_opt_in(ctx, k_block_fold<__nv_bfloat16>, smem, ctx->fs.attr_mask[9], 0)) return r;
-            k_block_fold<__nv_bfloat16><<<grid, kFoldWarps * 32, smem, st>>>(coefK, coefV, t_len, p->d_bins, wa, p->M, c.n_kv_heads, (uint32_t)c.n_dft);
+            k_block_fold<__nv_bfloat16><<<grid, kFoldWarps * 32, smem, st>>>(coefK, coefV, t_len, p->d_bins, wa, p->M, c.n_kv_heads, batch, (uint32_t)c.n_dft, splits);
         } else {
             if (int r = fft_opt_in(ctx, k_block_fold<float>, smem, ctx->fs.attr_mask[9], 1)) return r;
-            k_block_fold<float><<<grid, kFoldWarps * 32, smem, st>>>(coefK, coefV, t_len, p->d_bins, wa, p->M, c.n_kv_heads, (uint32_t)c.n_dft);
+            k_block_fold<float><<<grid, kFoldWarps * 32, smem, st>>>(coefK, coefV, t_len, p->d_bins, wa, p->M, c.n_kv_heads, batch, (uint32_t)c.n_dft, splits);
         }
         if (int r = launch_check(ctx, "k_block_fold")) return r;
         if (c.kv_dtype == FAEDKV_BF16)

@@ -58,9 +58,15 @@ __global__ void k_window_fill(const T *__restrict__ K, const T *__restrict__ V, 
 // exp(s - m), and o_w[col][c] = sum_w exp(s_w - m) v_w[c].  Rows: the S sink tokens, then the unfolded tokens
 // [S + folded(t + 1), t] in token order, where t = t_len is the step's new token; its ring slot is written only
 // at the end of the step, so k_new / v_new stand in for that row.  No rows at all: m = -inf, sum = 0, o = 0.
-// The host runs it on a second stream beside the first two FFT kernels, which leave the memory system idle:
-// beside a bandwidth-saturating pass its dependent loads would each cost many microseconds.
-// grid = (units, GQ): one CTA per query head; block = 256; dynamic smem = (S + Rc) floats.
+//
+// Nothing here depends on the rest of the step, so the host starts it on a second stream at the top of the
+// call, beside the pass over C_K, and joins it before the kernel that reads the statistics.  Beside a
+// bandwidth-saturating pass every dependent round of loads costs microseconds and every register held is one
+// the pass cannot use: a CTA is 128 threads of at most 64 registers and takes one query head; each of its 4
+// warps reads the K and V rows of kWinRows tokens at once (rows w = warp mod 4; kept in the storage type
+// until used) and runs an online softmax over them in registers (a lane holds 4 of the 128 channels); the
+// paper's window (60 rows; 110 with a deferred block of 50) takes 2 to 4 rounds.
+// grid = (units, GQ); block = 128.
 struct WindowArgs {
     const void *winK, *winV, *k_new, *v_new;   // storage type of the context
     int S, R, D, Rc;                           // sink, recent, defer block, ring capacity (win_ring(R, D))
@@ -68,172 +74,210 @@ struct WindowArgs {
     float *m_w, *s_w, *o_w;                    // statistics row of the window, [Gp] each; output [Gp][128]
 };
 
+template <typename T> struct WinRaw;
+template <> struct WinRaw<float> {
+    using type = float4;
+    static __device__ __forceinline__ type load(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+    static __device__ __forceinline__ float4 cvt(type r) { return r; }
+};
+template <> struct WinRaw<__nv_bfloat16> {
+    using type = uint2;
+    static __device__ __forceinline__ type load(const __nv_bfloat16 *p) { return *reinterpret_cast<const uint2 *>(p); }
+    static __device__ __forceinline__ float4 cvt(type r) {
+        return make_float4(bf16_bits_to_float(r.x & 0xffffu), __uint_as_float(r.x & 0xffff0000u),
+                           bf16_bits_to_float(r.y & 0xffffu), __uint_as_float(r.y & 0xffff0000u));
+    }
+};
+
+constexpr int kWinWarps = 4;                   // row shares of a query head
+
 template <typename TQ, int GQ>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kWinWarps * 32, 8)
 k_attn_window(const TQ *__restrict__ q, WindowArgs wa, const int32_t *__restrict__ t_len, int H) {
-    extern __shared__ float sc[];                     // [W] scores, then exp(s - m)
-    __shared__ float part[kHeadDim];
+    using Raw = WinRaw<TQ>;
+    constexpr int RS = kWinWarps;
+    constexpr int kWinRows = sizeof(TQ) == 2 ? 8 : 4;          // rows a warp has in flight
+    __shared__ float4 o_s[RS][32];
+    __shared__ float m_s[RS], s_s[RS];
     const TQ *winK = static_cast<const TQ *>(wa.winK), *winV = static_cast<const TQ *>(wa.winV);
     const TQ *k_new = static_cast<const TQ *>(wa.k_new), *v_new = static_cast<const TQ *>(wa.v_new);
     const int S = wa.S, Rc = wa.Rc, Wcap = S + Rc;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rs = warp;                                       // share of the rows
     const int bh = blockIdx.x, b = bh / H, col = bh * GQ + (int)blockIdx.y;     // one query head per CTA
+    const float4 qv = load4(q + (size_t)col * kHeadDim + lane * 4);
     const int t = t_len[b];
     const int first = win_folded(t + 1, S, wa.R, wa.D);       // offset (from S) of the oldest unfolded token
     const int W = S + (t + 1 - S - first);
-    // row w -> its row in the window tensor, or -1 for the step's new token
-    auto locate = [&](int w) { return w < S ? w : (first + w - S == t - S ? -1 : S + (first + w - S) % Rc); };
-    const float4 qv = load4(q + (size_t)col * kHeadDim + lane * 4);
-    // scores: a warp takes rows w = warp + 8u, all loads of a batch of 8 issued before any is used
-    for (int w0 = warp; w0 < W; w0 += 64) {
-        float4 kv[8];
+    const TQ *kbase = winK + (size_t)bh * Wcap * kHeadDim + lane * 4, *vbase = winV + (size_t)bh * Wcap * kHeadDim + lane * 4;
+    const TQ *kn = k_new + (size_t)bh * kHeadDim + lane * 4, *vn = v_new + (size_t)bh * kHeadDim + lane * 4;
+    float m_run = -INFINITY, sum = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int w0 = rs; w0 < W; w0 += RS * kWinRows) {
+        typename Raw::type kr[kWinRows], vr[kWinRows];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int w = w0 + 8 * u;
-            kv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (w < W) {
-                const int row = locate(w);
-                const TQ *krow = row < 0 ? k_new + (size_t)bh * kHeadDim : winK + ((size_t)bh * Wcap + row) * kHeadDim;
-                kv[u] = load4(krow + lane * 4);
-            }
+        for (int u = 0; u < kWinRows; ++u) {
+            const int w = min(w0 + RS * u, W - 1);   // rows past W repeat the last one; their scores are dropped
+            // row of the window tensor, or the step's new token
+            const int n = first + w - S;             // offset from S of an unfolded token (w >= S)
+            const bool is_new = w >= S && n == t - S;
+            const size_t off = (size_t)(w < S ? w : S + n % Rc) * kHeadDim;
+            kr[u] = Raw::load(is_new ? kn : kbase + off);
+            vr[u] = Raw::load(is_new ? vn : vbase + off);
         }
-        float d[8];
+        float d[kWinRows];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) d[u] = kv[u].x * qv.x + kv[u].y * qv.y + kv[u].z * qv.z + kv[u].w * qv.w;
+        for (int u = 0; u < kWinRows; ++u) {
+            const float4 k4 = Raw::cvt(kr[u]);
+            d[u] = k4.x * qv.x + k4.y * qv.y + k4.z * qv.z + k4.w * qv.w;
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-            for (int u = 0; u < 8; ++u) d[u] += __shfl_xor_sync(0xffffffffu, d[u], o);     // 8 independent chains
-        if (lane < 8 && w0 + 8 * lane < W) {
-            float v = d[0];
+            for (int u = 0; u < kWinRows; ++u) d[u] += __shfl_xor_sync(0xffffffffu, d[u], o);   // independent chains
+        float m_new = m_run;
 #pragma unroll
-            for (int u = 1; u < 8; ++u) v = lane == u ? d[u] : v;
-            sc[w0 + 8 * lane] = v * wa.scale;
+        for (int u = 0; u < kWinRows; ++u) {
+            d[u] = w0 + RS * u < W ? d[u] * wa.scale : -INFINITY;
+            m_new = fmaxf(m_new, d[u]);
         }
-    }
-    __syncthreads();
-    if (warp == 0) {
-        float m = -INFINITY;
-        for (int w = lane; w < W; w += 32) m = fmaxf(m, sc[w]);
+        const float f = m_run == -INFINITY ? 0.f : __expf(m_run - m_new);      // m_new is finite: row w0 exists
+        sum *= f;
+        acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        float sum = 0.f;
-        for (int w = lane; w < W; w += 32) {
-            const float p = __expf(sc[w] - m);
-            sc[w] = p;
+        for (int u = 0; u < kWinRows; ++u) {
+            const float p = __expf(d[u] - m_new);                              // 0 for the rows past W
+            const float4 v4 = Raw::cvt(vr[u]);
             sum += p;
+            acc.x = fmaf(p, v4.x, acc.x); acc.y = fmaf(p, v4.y, acc.y);
+            acc.z = fmaf(p, v4.z, acc.z); acc.w = fmaf(p, v4.w, acc.w);
         }
+        m_run = m_new;
+    }
+    // the row shares meet in shared memory
+    o_s[rs][lane] = acc;
+    if (lane == 0) {
+        m_s[rs] = m_run;
+        s_s[rs] = sum;
+    }
+    __syncthreads();
+    {
+        const int c = threadIdx.x;                             // 128 threads, 128 channels
+        float m = m_s[0];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        if (lane == 0) {
+        for (int r = 1; r < RS; ++r) m = fmaxf(m, m_s[r]);
+        float o = 0.f, sm = 0.f;
+#pragma unroll
+        for (int r = 0; r < RS; ++r) {
+            const float f = m_s[r] == -INFINITY ? 0.f : __expf(m_s[r] - m);
+            sm = fmaf(s_s[r], f, sm);
+            o = fmaf(reinterpret_cast<const float *>(&o_s[r][0])[c], f, o);
+        }
+        wa.o_w[(size_t)col * kHeadDim + c] = o;
+        if (c == 0) {
             wa.m_w[col] = m;
-            wa.s_w[col] = sum;
+            wa.s_w[col] = sm;
         }
     }
-    __syncthreads();
-    // output: thread (channel c, half) sums the rows of its parity, 8 loads in flight; halves meet in shared memory
-    const int c = threadIdx.x & (kHeadDim - 1), half = threadIdx.x >> 7;
-    float acc = 0.f;
-    for (int w0 = half; w0 < W; w0 += 16) {
-        float vv[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int w = w0 + 2 * u;
-            vv[u] = 0.f;
-            if (w < W) {
-                const int row = locate(w);
-                const TQ *vrow = row < 0 ? v_new + (size_t)bh * kHeadDim : winV + ((size_t)bh * Wcap + row) * kHeadDim;
-                vv[u] = load1(vrow + c);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (w0 + 2 * u < W) acc = fmaf(sc[w0 + 2 * u], vv[u], acc);
-    }
-    if (half == 1) part[c] = acc;
-    __syncthreads();
-    if (half == 0) wa.o_w[(size_t)col * kHeadDim + c] = acc + part[c];
 }
 
 // Block fold (Eq. 12 for D tokens at once): for every sequence whose token count reaches a block boundary with
 // this step's token, the D oldest unfolded tokens are folded into C_K and C_V at the next D positions of the
-// transformed segment, oldest first, with the very FMAs of D single-token updates (bit-identical planes).
-// The other sequences' CTAs return at once.  t_len is not changed here.
-// A warp owns kFoldBins bins at a time (a lane holds 4 of the 128 channels); the D tokens of the unit sit in
-// shared memory as float, the D twiddles of each bin are computed by the lanes and broadcast through shared
-// memory, so one token row read feeds kFoldBins * 8 FMAs.
-// grid = (ceil(M / (8 * kFoldBins)), units, 2 {K, V}); block = 256;
-// dynamic smem = D * 128 floats + 8 warps * kFoldBins * D float2.
-constexpr int kFoldBins = 4;
+// transformed segment, oldest first, with the very FMAs of D single-token updates (bit-identical planes:
+// x * (-s) is -(x * s) exactly).  t_len is not changed.
+//
+// Work items are (sequence, group of 64 bins, share of the 2H {kv head, K or V} planes), dealt round-robin to a
+// grid of a few CTAs per SM; items of sequences that do not fold this step cost one look at t_len, so the
+// launch is nearly free on the steps without a fold.  Per item the 64 x D twiddles are computed once (they
+// depend on bin and position only) and kept in shared memory as (c, -s), token-major; per plane the D token rows
+// are staged as float, then each warp owns 8 bins (a lane holds 4 of the 128 channels): per token one 16-byte
+// read of the token row and four 16-byte broadcast reads of twiddles, all at fixed offsets from one running
+// pointer each, feed 64 FMAs -- the kernel is bound by FMA issue, not by HBM.
+// grid = (n_ctas); block = 256; dynamic smem = block_fold_smem(D).
+constexpr int kFoldBins = 8;                       // bins per warp
 constexpr int kFoldWarps = 8;
+constexpr int kFoldGroup = kFoldBins * kFoldWarps; // bins per work item
 inline size_t block_fold_smem(int D) {
-    return (size_t)D * kHeadDim * sizeof(float) + (size_t)kFoldWarps * kFoldBins * D * sizeof(float2);
+    return (size_t)D * kHeadDim * sizeof(float) + (size_t)kFoldGroup * D * sizeof(float2);
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kFoldWarps * 32)
+__global__ void __launch_bounds__(kFoldWarps * 32, 2)
 k_block_fold(float *__restrict__ coefK, float *__restrict__ coefV, const int32_t *__restrict__ t_len,
-             const int32_t *__restrict__ bins, WindowArgs wa, int M, int H, uint32_t P) {
+             const int32_t *__restrict__ bins, WindowArgs wa, int M, int H, int batch, uint32_t P, int splits) {
     extern __shared__ __align__(16) unsigned char fold_smem[];
     const int S = wa.S, R = wa.R, D = wa.D, Rc = wa.Rc;
-    const int unit = blockIdx.y, b = unit / H, kv = blockIdx.z;
-    const int t = t_len[b];
-    const int cnt = t + 1 - S - R;                   // unfolded tokens beyond the recent window, with the new one
-    if (cnt <= 0 || cnt % D != 0) return;
-    const int first = cnt - D;                       // tokens already folded = position of the oldest unfolded one
-    float *xs = reinterpret_cast<float *>(fold_smem);                                        // [D][128]
-    float2 *tws = reinterpret_cast<float2 *>(fold_smem + (size_t)D * kHeadDim * sizeof(float));
-    const T *win = static_cast<const T *>(kv == 0 ? wa.winK : wa.winV);
-    const T *x_new = static_cast<const T *>(kv == 0 ? wa.k_new : wa.v_new);
-    for (int e = threadIdx.x; e < D * kHeadDim; e += blockDim.x) {
-        const int i = e / kHeadDim, c = e % kHeadDim;
-        const int n = first + i;                     // token S + n
-        const T *row = (S + n == t) ? x_new + (size_t)unit * kHeadDim
-                                    : win + ((size_t)unit * (S + Rc) + S + n % Rc) * kHeadDim;
-        xs[e] = load1(row + c);
-    }
-    __syncthreads();
+    float *xs = reinterpret_cast<float *>(fold_smem);                                                    // [D][128]
+    float2 *tws = reinterpret_cast<float2 *>(fold_smem + (size_t)D * kHeadDim * sizeof(float));          // [D][64]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float2 *twl = tws + (size_t)warp * kFoldBins * D;
+    const int n_groups = (M + kFoldGroup - 1) / kFoldGroup, combos = 2 * H, per_split = (combos + splits - 1) / splits;
+    const int n_items = batch * n_groups * splits;
     const size_t plane = (size_t)M * kHeadDim;
-    float *base = (kv == 0 ? coefK : coefV) + (size_t)unit * 2 * plane;
-    const int k0 = (blockIdx.x * kFoldWarps + warp) * kFoldBins;
-    if (k0 >= M) return;
-    const int nb = min(kFoldBins, M - k0);
-    for (int e = lane; e < nb * D; e += 32) {
-        const int j = e / D, i = e % D;
-        float cs, sn;
-        twiddle(phase_mod((uint32_t)bins[k0 + j], (uint32_t)(first + i) % P, P), P, cs, sn);
-        twl[j * D + i] = make_float2(cs, sn);
-    }
-    float4 re[kFoldBins], im[kFoldBins];
-#pragma unroll
-    for (int j = 0; j < kFoldBins; ++j) {
-        re[j] = im[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j < nb) {
-            const float *rp = base + (size_t)(k0 + j) * kHeadDim + lane * 4;
-            re[j] = ld_stream(rp);
-            im[j] = ld_stream(rp + plane);
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const int sp = item % splits, grp = (item / splits) % n_groups, b = item / (splits * n_groups);
+        const int t = t_len[b];
+        const int cnt = t + 1 - S - R;               // unfolded tokens beyond the recent window, with the new one
+        if (cnt <= 0 || cnt % D != 0) continue;      // the whole CTA agrees: t depends on the sequence only
+        const int first = cnt - D;                   // tokens already folded = position of the oldest waiting one
+        const int k0 = grp * kFoldGroup;
+        __syncthreads();                             // the previous item's tables are no longer read
+        for (int e = threadIdx.x; e < kFoldGroup * D; e += blockDim.x) {
+            const int i = e / kFoldGroup, j = e % kFoldGroup;
+            float cs, sn;                            // columns past the last bin repeat it; nothing stores their results
+            twiddle(phase_mod((uint32_t)bins[min(k0 + j, M - 1)], (uint32_t)(first + i) % P, P), P, cs, sn);
+            tws[e] = make_float2(cs, -sn);
         }
-    }
-    __syncwarp();
-    for (int i = 0; i < D; ++i) {
-        const float4 x = *reinterpret_cast<const float4 *>(xs + i * kHeadDim + lane * 4);
+        const int kb = k0 + warp * kFoldBins, nb = max(0, min(kFoldBins, M - kb));
+        for (int cb = sp * per_split; cb < min(combos, (sp + 1) * per_split); ++cb) {
+            const int unit = b * H + (cb >> 1), kv = cb & 1;
+            const T *win = static_cast<const T *>(kv == 0 ? wa.winK : wa.winV);
+            const T *x_new = static_cast<const T *>(kv == 0 ? wa.k_new : wa.v_new);
+            __syncthreads();                         // the previous plane's token rows are no longer read
+            for (int i = warp; i < D; i += kFoldWarps) {
+                const int n = first + i;             // token S + n
+                const T *row = (S + n == t) ? x_new + (size_t)unit * kHeadDim
+                                            : win + ((size_t)unit * (S + Rc) + S + n % Rc) * kHeadDim;
+                *reinterpret_cast<float4 *>(xs + i * kHeadDim + lane * 4) = load4(row + lane * 4);
+            }
+            __syncthreads();
+            if (nb == 0) continue;
+            float *base = (kv == 0 ? coefK : coefV) + (size_t)unit * 2 * plane;
+            float4 re[kFoldBins], im[kFoldBins];
 #pragma unroll
-        for (int j = 0; j < kFoldBins; ++j) {
-            const float2 cs = twl[j * D + i];        // rows past nb hold stale values; their results are dropped
-            re[j].x = fmaf(x.x, cs.x, re[j].x); im[j].x = fmaf(-x.x, cs.y, im[j].x);
-            re[j].y = fmaf(x.y, cs.x, re[j].y); im[j].y = fmaf(-x.y, cs.y, im[j].y);
-            re[j].z = fmaf(x.z, cs.x, re[j].z); im[j].z = fmaf(-x.z, cs.y, im[j].z);
-            re[j].w = fmaf(x.w, cs.x, re[j].w); im[j].w = fmaf(-x.w, cs.y, im[j].w);
-        }
-    }
+            for (int j = 0; j < kFoldBins; ++j) {
+                re[j] = im[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (j < nb) {
+                    const float *rp = base + (size_t)(kb + j) * kHeadDim + lane * 4;
+                    re[j] = ld_stream(rp);
+                    im[j] = ld_stream(rp + plane);
+                }
+            }
+            const float4 *tp = reinterpret_cast<const float4 *>(tws + warp * kFoldBins);   // two bins' (c, -s) per read
+            const float4 *xp = reinterpret_cast<const float4 *>(xs) + lane;
+#pragma unroll 2
+            for (int i = 0; i < D; ++i, tp += kFoldGroup / 2, xp += kHeadDim / 4) {
+                const float4 x = *xp;
 #pragma unroll
-    for (int j = 0; j < kFoldBins; ++j) {
-        if (j < nb) {
-            float *wp = base + (size_t)(k0 + j) * kHeadDim + lane * 4;
-            st_stream(wp, re[j]);
-            st_stream(wp + plane, im[j]);
+                for (int j = 0; j < kFoldBins; j += 2) {
+                    const float4 w = tp[j / 2];
+                    re[j].x = fmaf(x.x, w.x, re[j].x); im[j].x = fmaf(x.x, w.y, im[j].x);
+                    re[j].y = fmaf(x.y, w.x, re[j].y); im[j].y = fmaf(x.y, w.y, im[j].y);
+                    re[j].z = fmaf(x.z, w.x, re[j].z); im[j].z = fmaf(x.z, w.y, im[j].z);
+                    re[j].w = fmaf(x.w, w.x, re[j].w); im[j].w = fmaf(x.w, w.y, im[j].w);
+                    re[j + 1].x = fmaf(x.x, w.z, re[j + 1].x); im[j + 1].x = fmaf(x.x, w.w, im[j + 1].x);
+                    re[j + 1].y = fmaf(x.y, w.z, re[j + 1].y); im[j + 1].y = fmaf(x.y, w.w, im[j + 1].y);
+                    re[j + 1].z = fmaf(x.z, w.z, re[j + 1].z); im[j + 1].z = fmaf(x.z, w.w, im[j + 1].z);
+                    re[j + 1].w = fmaf(x.w, w.z, re[j + 1].w); im[j + 1].w = fmaf(x.w, w.w, im[j + 1].w);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < kFoldBins; ++j) {
+                if (j < nb) {
+                    float *wp = base + (size_t)(kb + j) * kHeadDim + lane * 4;
+                    st_stream(wp, re[j]);
+                    st_stream(wp + plane, im[j]);
+                }
+            }
         }
     }
 }
