@@ -186,3 +186,57 @@ def test_config4_sweep_cells(fk, oracle, T, B, r, mask_kind, layer):
     (T, batch, retention, mask) sweep, one layer each, prefill + 32 decode steps."""
     _decode_case(fk, oracle, config=4, layer=layer, B=B, H=32, HQ=32, T=T, M=T // r, mask_kind=mask_kind,
                  steps=32, sample_units=[(B - 1, 17)], sample_steps=[31])
+
+
+@pytest.mark.parametrize("defer", [1, 50])
+def test_config2_windowed_workflow(fk, oracle, defer):
+    """configs[2] shape through the paper's own workflow (sink 10 + recent 50), per-step fold and
+    block-deferred fold of 50 tokens: one layer at full size, 110 decode steps (the deferred form folds
+    at steps 25 and 75), sampled units against the oracle's WindowedUnit at steps around the folds."""
+    from paper_2507_20030_b200 import synth
+    config, layer, B, H, HQ, T, M, S, R, steps = 2, 3, 16, 8, 32, 16384, 2048, 10, 50, 110
+    sample_units, sample_steps = [(0, 1), (13, 6)], [25, 26, 109]
+    P, GQ = T, HQ // H
+    seed = synth.config_seed(config)
+    ctx = fk.Context(n_layers=layer + 1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=fk.BF16,
+                     n_sink=S, n_recent=R, n_defer=defer)
+    mask = fk.mask_mixed(P, M, layer, seed)
+    ctx.plan(layer, mask)
+    bins = oracle.plan(P, oracle.mask_mixed(P, M, layer, seed))
+    assert ctx.get_bins(layer).tobytes() == bins.tobytes()
+    lseed = synth.config_seed(config, layer)
+    K, V = synth.make_kv(lseed, B, H, T, D, dtype=torch.bfloat16, device="cuda")
+    Kn, Vn = synth.make_kv(lseed, B, H, steps, D, pos0=T, dtype=torch.bfloat16, device="cuda", stream_tag=1)
+    units = {}
+    for b, h in sample_units:
+        u = units[(b, h)] = oracle.WindowedUnit(P, bins, S, R, defer=defer)
+        u.prefill(to_np64(K[b, h].cpu()), to_np64(V[b, h].cpu()))
+    cK, cV = ctx.alloc_coef(layer, B), ctx.alloc_coef(layer, B)
+    wK, wV = ctx.alloc_window(B), ctx.alloc_window(B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.prefill_windowed(layer, K, V, cK, cV, wK, wV, t_len)
+    out = torch.empty((B, HQ, D), dtype=torch.bfloat16, device="cuda")
+    folds = 0
+    for s in range(steps):
+        k_new, v_new = Kn[:, :, s].contiguous(), Vn[:, :, s].contiguous()
+        q = synth.make_q(lseed, s, B, HQ, D, dtype=torch.bfloat16, device="cuda")
+        ctx.step_windowed(layer, k_new, v_new, q, cK, cV, wK, wV, t_len, out)
+        for (b, h), u in units.items():
+            before = u.folded
+            u.step(to_np64(k_new[b, h].cpu()), to_np64(v_new[b, h].cpu()))
+            folds += (u.folded - before) >= max(defer, 2)
+        if s in sample_steps:
+            got = to_np64(out)
+            for (b, h), u in units.items():
+                want = u.attention(to_np64(q[b, h * GQ:(h + 1) * GQ].cpu()))
+                err = np.abs(got[b, h * GQ:(h + 1) * GQ] - want).max()
+                assert err <= ATTN_MAX_ABS, ("attention", s, b, h, err)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0 and t_len.tolist() == [T + steps] * B
+    assert folds == (2 * len(sample_units) if defer > 1 else 0)
+    for (b, h), u in units.items():
+        assert u.folded == (T + steps - S - R) // defer * defer
+        for c, want in ((cK, u.CK), (cV, u.CV)):
+            err = rel_l2(to_np64(c[b, h]), np.stack(want))
+            assert err <= REL_L2_BF16, ("planes", b, h, err)
+    ctx.close()
