@@ -75,8 +75,10 @@ typedef enum {
                                 bf16 tensors: tensor-core path; float32 tensors: float32 SIMT path */
     FAEDKV_DECODE_SIMT = 1,  /* float32 FMA contractions, twiddles exact to float32            */
     FAEDKV_DECODE_UMMA = 2,  /* tcgen05 contractions with f16 operands, float32 accumulate (bf16 tensors only) */
-    FAEDKV_DECODE_FFT = 3    /* float32 two-pass shared-memory FFTs (power-of-two P only): O(P log P) per
+    FAEDKV_DECODE_FFT = 3,   /* float32 shared-memory FFTs (power-of-two P only; one kernel per column for
+                                P <= 16384, two passes through an L2-resident array above): O(P log P) per
                                 query head instead of O(P * M)                                 */
+    FAEDKV_DECODE_FFT_TWO_PASS = 4  /* FAEDKV_DECODE_FFT restricted to the two-pass kernels at every P */
 } faedkv_decode_mode;
 
 typedef struct {

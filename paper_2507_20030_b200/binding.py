@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "lib", "libfaedkv.so")
 F32, BF16 = 0, 1
 PREFILL_AUTO, PREFILL_SIMT, PREFILL_UMMA, PREFILL_FFT = 0, 1, 2, 3
 STATE_SUM, STATE_MEAN, STATE_ROTATING = 0, 1, 2
-DECODE_AUTO, DECODE_SIMT, DECODE_UMMA, DECODE_FFT = 0, 1, 2, 3
+DECODE_AUTO, DECODE_SIMT, DECODE_UMMA, DECODE_FFT, DECODE_FFT_TWO_PASS = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "faedkv_create", "faedkv_destroy", "faedkv_last_error", "faedkv_plan", "faedkv_n_bins",

@@ -18,6 +18,7 @@
 #include "k_idft_umma.cuh"
 #include "k_attn_umma.cuh"
 #include "k_attn_fft.cuh"
+#include "k_attn_col.cuh"
 #include "k_recon_fft.cuh"
 #include "k_prefill_fft.cuh"
 #include "k_ablate.cuh"
@@ -52,11 +53,13 @@ struct FftScratch {
     int recon_units = 0;                  // units (sequence, kv head) per launch group of the reconstruction
     float *mloc = nullptr, *sloc = nullptr, *colsum = nullptr;   // [N1 + 1][Gp] (last row: the window), [2][Gp]
     float *o_win = nullptr;               // [Gp][128] unnormalised attention output over the sink + recent window
+    float2 *Wg = nullptr;                 // [Gp][max_M] probability-spectrum weights (one-kernel column transform)
+    float2 *colE = nullptr, *colB = nullptr, *colP = nullptr;   // its twiddle tables (see k_col_tables)
     cudaStream_t side = nullptr;          // second stream: the window kernel runs beside the FFT kernels
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     unsigned int *tickets = nullptr;      // [max_batch * H + max_batch], zero between calls
     int max_M = 0;
-    unsigned int attr_mask[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
+    unsigned int attr_mask[11] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
 };
 
 }  // namespace
@@ -78,6 +81,7 @@ struct faedkv_ctx {
     TcScratch tc;
     bool use_tc = false;               // bf16 tensors and decode_mode != SIMT
     bool use_fft = false;              // power-of-two P: FFT-shaped transforms in decode attention and reconstruction
+    bool use_col = false;              // ... and P <= 16384: decode attention's transforms as one kernel per column
     bool prefill_fft = false;          // FFT-shaped prefill transform
     FftScratch fs;
     unsigned long long launches = 0;   // kernels enqueued by this context so far
@@ -161,7 +165,7 @@ void free_scratch(faedkv_ctx *ctx) {
     cudaFree(t.cmax); cudaFree(t.psum); cudaFree(t.colsum); cudaFree(t.PfS);
     t = TcScratch();
     FftScratch &f = ctx->fs;
-    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.o_win); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr);
+    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.o_win); cudaFree(f.Wg); cudaFree(f.colE); cudaFree(f.colB); cudaFree(f.colP); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr);
     if (f.side != nullptr) cudaStreamDestroy(f.side);
     if (f.ev_fork != nullptr) cudaEventDestroy(f.ev_fork);
     if (f.ev_join != nullptr) cudaEventDestroy(f.ev_join);
@@ -223,10 +227,18 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             if (ctx->prefill_fft) CUDA_TRY(ctx, cudaMalloc(&f.Zr, ru * unit_bytes));
         }
         if (M > f.max_M) {
-            cudaFree(f.Qs);
-            f.Qs = nullptr;
+            cudaFree(f.Qs); cudaFree(f.Wg);
+            f.Qs = f.Wg = nullptr;
             CUDA_TRY(ctx, cudaMalloc(&f.Qs, (size_t)M * g.Gp * sizeof(float2)));
+            if (ctx->use_col) CUDA_TRY(ctx, cudaMalloc(&f.Wg, (size_t)M * g.Gp * sizeof(float2)));
             f.max_M = M;
+        }
+        if (ctx->use_col && f.colE == nullptr) {
+            CUDA_TRY(ctx, cudaMalloc(&f.colE, sizeof(float2) << colfft::kLgE));
+            CUDA_TRY(ctx, cudaMalloc(&f.colB, sizeof(float2) << colfft::kLgE));
+            CUDA_TRY(ctx, cudaMalloc(&f.colP, sizeof(float2) * ((size_t)g.N + 1)));
+            colfft::k_col_tables<<<32, 256>>>(f.colE, f.colB, f.colP, (uint32_t)c.n_dft);
+            CUDA_TRY(ctx, cudaDeviceSynchronize());
         }
     }
     if (ctx->use_tc) {
@@ -602,10 +614,37 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
         k_attn_qs<TQ, GQ, APPEND><<<grid, kAttnWarps * 32, 0, st>>>(
             static_cast<const TQ *>(q), coefK, static_cast<const TQ *>(foldK), t_len, p.d_bins, f.Qs, M, H, HQ, g.Gp,
-            (uint32_t)P, scale / (float)P, fold);
+            (uint32_t)P, scale / (float)P, fold, ctx->use_col ? 1 : 0);
         if (int r = launch_check(ctx, "k_attn_qs")) return r;
     }
     int rc = FAEDKV_ERR_UNSUPPORTED;
+    if (ctx->use_col) {
+        // steps (2)-(4) in one kernel: a CTA per column holds the whole packed signal in shared memory
+        if (n_extra) CUDA_TRY(ctx, cudaStreamWaitEvent(st, f.ev_join, 0));
+        const int n_tiles = g.N1 >> lgMT;
+        const float *m_w = n_extra ? f.mloc + (size_t)n_tiles * g.Gp : nullptr, *s_w = n_extra ? f.sloc + (size_t)n_tiles * g.Gp : nullptr;
+#define CALL(LG)                                                                                         \
+        rc = fft_opt_in(ctx, colfft::k_afft_col<LG>, colfft::smem_bytes<LG>(), f.attr_mask[10], LG);      \
+        if (rc == 0) launch_pdl(colfft::k_afft_col<LG>, dim3(batch * HQ), dim3(colfft::threads<LG>()), colfft::smem_bytes<LG>(), st, \
+                                (uint32_t)P, M, p.d_slot, p.d_bins, f.Qs, f.colE, f.colB, f.colP, t_len, HQ,        \
+                                (counts_new ? 1 : 0) - S - R, D, m_w, s_w, f.Wg, f.colsum, g.Gp)
+        switch (g.lgN1 + g.lgN2) {
+            case 5: CALL(5); break;
+            case 6: CALL(6); break;
+            case 7: CALL(7); break;
+            case 8: CALL(8); break;
+            case 9: CALL(9); break;
+            case 10: CALL(10); break;
+            case 11: CALL(11); break;
+            case 12: CALL(12); break;
+            case 13: CALL(13); break;
+            default: break;
+        }
+#undef CALL
+        if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no column kernel for 2^%d points", g.lgN1 + g.lgN2) : rc;
+        if (int r = launch_check(ctx, "k_afft_col")) return r;
+    } else {
+    rc = FAEDKV_ERR_UNSUPPORTED;
     {
         const dim3 grid(g.N2 >> lgKT, col_blocks);
         const size_t smem = afft_smem_a(g.lgN1, lgKT, true);
@@ -642,6 +681,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN1) : rc;
         if (int r = launch_check(ctx, "k_afft_fwd_b")) return r;
     }
+    }
     {
         const int slices = out_slices(ctx, batch, M);
         const int per = (M + slices - 1) / slices;
@@ -649,7 +689,8 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         launch_pdl(k_attn_out_fft<TQ, GQ, APPEND>, grid, dim3(kAttnWarps * 32), 0, st,
                    coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
                    static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, counts_new ? 1 : 0,
-                   windowed ? WindowArgs{winK, winV, k_new, v_new, S, R, D, Rc, 0.f, nullptr, nullptr, nullptr} : WindowArgs{});
+                   windowed ? WindowArgs{winK, winV, k_new, v_new, S, R, D, Rc, 0.f, nullptr, nullptr, nullptr} : WindowArgs{},
+                   ctx->use_col ? f.Wg : nullptr);
         if (int r = launch_check(ctx, "k_attn_out_fft")) return r;
     }
     return FAEDKV_OK;
@@ -831,9 +872,10 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     if (cfg->kv_dtype != FAEDKV_F32 && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->prefill_mode < FAEDKV_PREFILL_AUTO || cfg->prefill_mode > FAEDKV_PREFILL_FFT) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->twiddle_terms < 0 || cfg->twiddle_terms > 2) return FAEDKV_ERR_INVALID_ARG;
-    if (cfg->decode_mode < FAEDKV_DECODE_AUTO || cfg->decode_mode > FAEDKV_DECODE_FFT) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->decode_mode < FAEDKV_DECODE_AUTO || cfg->decode_mode > FAEDKV_DECODE_FFT_TWO_PASS) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->decode_mode == FAEDKV_DECODE_UMMA && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_UNSUPPORTED;
-    if (cfg->decode_mode == FAEDKV_DECODE_FFT && !fft::supported(cfg->n_dft)) return FAEDKV_ERR_UNSUPPORTED;
+    if ((cfg->decode_mode == FAEDKV_DECODE_FFT || cfg->decode_mode == FAEDKV_DECODE_FFT_TWO_PASS) && !fft::supported(cfg->n_dft))
+        return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_sink < 0 || cfg->n_recent < 0 || cfg->n_sink + cfg->n_recent > 1024) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->n_defer < 0 || cfg->n_defer > 128) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->head_dim != kHeadDim) return FAEDKV_ERR_UNSUPPORTED;
@@ -849,8 +891,10 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     ctx->hqp = (cfg->n_q_heads + 31) / 32 * 32;
     ctx->use_tc = cfg->kv_dtype == FAEDKV_BF16 && cfg->decode_mode != FAEDKV_DECODE_SIMT;
     const bool fft_ok = fft::supported(cfg->n_dft) && fft::fits_32bit_index(cfg->n_dft, cfg->max_batch * cfg->n_q_heads);
-    if (cfg->decode_mode == FAEDKV_DECODE_FFT && !fft_ok) { delete ctx; return FAEDKV_ERR_UNSUPPORTED; }
-    ctx->use_fft = fft_ok && (cfg->decode_mode == FAEDKV_DECODE_AUTO || cfg->decode_mode == FAEDKV_DECODE_FFT);
+    const bool fft_mode = cfg->decode_mode == FAEDKV_DECODE_FFT || cfg->decode_mode == FAEDKV_DECODE_FFT_TWO_PASS;
+    if (fft_mode && !fft_ok) { delete ctx; return FAEDKV_ERR_UNSUPPORTED; }
+    ctx->use_fft = fft_ok && (cfg->decode_mode == FAEDKV_DECODE_AUTO || fft_mode);
+    ctx->use_col = ctx->use_fft && cfg->decode_mode != FAEDKV_DECODE_FFT_TWO_PASS && cfg->n_dft <= (2 << colfft::kMaxLg);
     // the FFT-shaped prefill shares the decode path's scratch, so it needs that path too
     if (cfg->prefill_mode == FAEDKV_PREFILL_FFT && !ctx->use_fft) { delete ctx; return FAEDKV_ERR_UNSUPPORTED; }
     ctx->prefill_fft = ctx->use_fft && (cfg->prefill_mode == FAEDKV_PREFILL_FFT ||

@@ -27,7 +27,7 @@ template <typename TQ, int GQ, bool APPEND>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restrict__ k_new,
           const int32_t *__restrict__ t_len, const int32_t *__restrict__ bins, float2 *__restrict__ Qs,
-          int M, int H, int HQ, int Gp, uint32_t P, float scale_over_P, FoldSrc fold) {
+          int M, int H, int HQ, int Gp, uint32_t P, float scale_over_P, FoldSrc fold, int col_major) {
     constexpr int KB = 16 / GQ;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -85,7 +85,9 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
         const uint32_t bin = (uint32_t)bins[k0 + kk];
         // bins 0 and P/2 are their own mirrors: only their real part enters a real signal
         const bool self_conj = bin == 0u || 2u * bin == P;
-        float *dst = reinterpret_cast<float *>(Qs + (size_t)(k0 + kk) * Gp + b * HQ + h * GQ + g);
+        // Qs[bin][col] for the two-pass transforms, Qs[col][bin] for the one-kernel column transform
+        const size_t col = (size_t)(b * HQ + h * GQ + g);
+        float *dst = reinterpret_cast<float *>(Qs + (col_major ? col * M + (k0 + kk) : (size_t)(k0 + kk) * Gp + col));
         dst[pl] = (pl == 1 && self_conj) ? 0.f : tot * scale_over_P;
     }
 }
@@ -345,7 +347,7 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
                const float2 *__restrict__ Zf, const float *__restrict__ colsum, const int32_t *__restrict__ bins,
                float *__restrict__ partial, unsigned int *__restrict__ tickets, TQ *__restrict__ out,
                int M, int H, int HQ, fft::Geometry g, int bins_per_slice, float inv_P, FoldSrc fold,
-               const float *__restrict__ o_win, int bump, WindowArgs commit) {
+               const float *__restrict__ o_win, int bump, WindowArgs commit, const float2 *__restrict__ Wg) {
     using namespace fft;
     // the weights of a chunk and the final cross-warp reduction share one buffer
     constexpr size_t kWgtBytes = (size_t)kOutChunk * GQ * sizeof(float2) + (APPEND ? kOutChunk * sizeof(float2) : 0);
@@ -377,7 +379,16 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
     for (int c0 = kbeg; c0 < kend; c0 += kOutChunk) {
         const int cn = min(kOutChunk, kend - c0);
         __syncthreads();                             // previous chunk's weights are no longer read
-        if ((int)threadIdx.x < cn) {
+        if ((int)threadIdx.x < cn && Wg != nullptr) {
+            // the column transform has left the weights ready: Wg[col][bin index]
+#pragma unroll
+            for (int q = 0; q < GQ; ++q) wgt[threadIdx.x][q] = Wg[(size_t)(gcol + q) * M + c0 + threadIdx.x];
+            if (APPEND) {
+                float cs, sn;
+                twiddle(phase_mod((uint32_t)bins[c0 + threadIdx.x], t, g.P), g.P, cs, sn);
+                upd[threadIdx.x] = make_float2(cs, sn);
+            }
+        } else if ((int)threadIdx.x < cn) {
             const uint32_t bin = (uint32_t)bins[c0 + threadIdx.x];
             const float w = 0.5f * hermitian_weight(bin, g.P);
             const int ka = (int)bin & (g.N - 1), kb = (g.N - ka) & (g.N - 1);

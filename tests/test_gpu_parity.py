@@ -270,7 +270,8 @@ def _decode_modes(fk, dtype, P):
     if dtype == torch.bfloat16:
         modes.append(fk.DECODE_UMMA)
     if P & (P - 1) == 0 and P >= 64:
-        modes.append(fk.DECODE_FFT)
+        modes.append(fk.DECODE_FFT)               # one kernel per column up to P = 16384
+        modes.append(fk.DECODE_FFT_TWO_PASS)      # the two-pass kernels, which larger grids use
     return modes
 
 
@@ -329,7 +330,8 @@ def test_decode_attn_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, tl, vs
         ctx.close()
 
 
-@pytest.mark.parametrize("P,M,B,H,HQ", [(32768, 48, 1, 2, 8), (131072, 32, 2, 1, 4), (16384, 64, 3, 2, 4)])
+@pytest.mark.parametrize("P,M,B,H,HQ", [(32768, 48, 1, 2, 8), (131072, 32, 2, 1, 4), (16384, 64, 3, 2, 4),
+                                         (8192, 64, 2, 2, 2), (4096, 32, 2, 1, 8)])
 def test_decode_attn_fft_long_grids(fk, oracle, P, M, B, H, HQ):
     """FFT-shaped transforms at the grid sizes of the long-context workloads (few bins, so that the
     oracle's materialised reconstruction stays cheap); ragged live lengths."""
