@@ -15,8 +15,9 @@
 //
 // A stage is "every thread reads the inputs of its butterflies into registers; barrier; every thread writes
 // its outputs; barrier", which makes the autosort work in place.  Twiddles: a stage whose span NS * R is at
-// most 1024 looks them up in E[i] = e^{+j 2 pi i / 1024}; the last stage of a longer column (span = N) takes
-// w = e^{+j 2 pi k / N} from a second table and multiplies its way through w^2, w^3, ... (15 products at most).
+// most 1024 has a table of its own, laid out so that consecutive threads read consecutive entries (a shared
+// table indexed k * r is read with strides and bank conflicts); the last stage of a longer column (span = N)
+// takes w = e^{+j 2 pi k / N} from a table and multiplies its way through w^2, w^3, ... (15 products at most).
 // The column is padded by one element per 16 so that the stride-R writes of the first stage spread over
 // the banks.
 #pragma once
@@ -45,14 +46,21 @@ template <> struct Stages<13> { static constexpr int R1 = 8, R2 = 8, R3 = 8, R4 
 template <int LGN> __host__ __device__ constexpr int threads() {
     return (1 << LGN) / 16 < 64 ? 64 : ((1 << LGN) / 16 > 512 ? 512 : (1 << LGN) / 16);
 }
-// Entries of the w = e^{+j 2 pi k / N} table the last stage needs (0: every stage looks up E).
+// Entries of the w = e^{+j 2 pi k / N} table the last stage needs (0: every stage has a table of its own).
 template <int LGN> __host__ __device__ constexpr int chain_entries() {
     using S = Stages<LGN>;
     return (1 << LGN) <= (1 << kLgE) ? 0 : (1 << LGN) / (S::R4 > 1 ? S::R4 : (S::R3 > 1 ? S::R3 : S::R2));
 }
+// Entries of the per-stage twiddle tables tw[(r - 1) * NS + k] = e^{+j 2 pi k r / (NS * R)} of stages 2 and 3
+// (stage 3: 0 when it is the chained last stage, or absent).
+template <int LGN> __host__ __device__ constexpr int tw2_entries() { return (Stages<LGN>::R2 - 1) * Stages<LGN>::R1; }
+template <int LGN> __host__ __device__ constexpr int tw3_entries() {
+    using S = Stages<LGN>;
+    return (S::R3 > 1 && S::R1 * S::R2 * S::R3 <= (1 << kLgE)) ? (S::R3 - 1) * S::R1 * S::R2 : 0;
+}
 __host__ __device__ constexpr int padded(int idx) { return idx + (idx >> 4); }
 template <int LGN> constexpr size_t smem_bytes() {
-    return (size_t)(padded(1 << LGN) + 1 + (1 << kLgE) + chain_entries<LGN>()) * sizeof(float2);
+    return (size_t)(padded(1 << LGN) + 1 + tw2_entries<LGN>() + tw3_entries<LGN>() + chain_entries<LGN>()) * sizeof(float2);
 }
 
 // One in-place stage of radix R over the N-point column z; NS = product of the radices already applied.
@@ -61,8 +69,14 @@ template <int LGN> constexpr size_t smem_bytes() {
 // the low four bits of the base and of the offset never carry (NB and NS are multiples of 16, or base and
 // offset occupy disjoint low bits), so padded(base + offset) = padded(base) + padded(offset): one padded
 // base per butterfly, compile-time offsets from it.
-template <int N, int NT, int R, int NS, bool OWN, typename In>
-__device__ __forceinline__ void stage(float2 *__restrict__ z, const float2 *__restrict__ E, const float2 *__restrict__ Bt, In in) {
+// pre(value, index) is applied to every input read from the column, post(index, value) sees every output.
+struct NoPre { __device__ __forceinline__ float2 operator()(float2 v, int) const { return v; } };
+struct NoPost { __device__ __forceinline__ void operator()(int, float2) const {} };
+
+// tw: this stage's table tw[(r - 1) * NS + k] (consecutive threads read consecutive entries), or, for the
+// chained last stage of a long column, w[k] = e^{+j 2 pi k / N}.
+template <int N, int NT, int R, int NS, bool OWN, typename In, typename Pre, typename Post>
+__device__ __forceinline__ void stage(float2 *__restrict__ z, const float2 *__restrict__ tw, In in, Pre pre, Post post) {
     using namespace fft;
     constexpr int NB = N / R;                        // butterflies; also the stride of a butterfly's inputs
     constexpr int BPT = (NB + NT - 1) / NT;          // butterflies per thread
@@ -75,7 +89,7 @@ __device__ __forceinline__ void stage(float2 *__restrict__ z, const float2 *__re
         if constexpr (OWN) {
             const float2 *src = z + padded(j);
 #pragma unroll
-            for (int r = 0; r < R; ++r) v[b][r] = src[padded(r * NB)];
+            for (int r = 0; r < R; ++r) v[b][r] = pre(src[padded(r * NB)], j + r * NB);
         } else {
 #pragma unroll
             for (int r = 0; r < R; ++r) v[b][r] = in(j + r * NB);
@@ -83,11 +97,10 @@ __device__ __forceinline__ void stage(float2 *__restrict__ z, const float2 *__re
         if (NS > 1) {
             const int k = j & (NS - 1);
             if constexpr (T <= (1 << kLgE)) {
-                const float2 *tw = E + k * ((1 << kLgE) / T);
 #pragma unroll
-                for (int r = 1; r < R; ++r) v[b][r] = cmul(v[b][r], tw[(r - 1) * k * ((1 << kLgE) / T)]);
+                for (int r = 1; r < R; ++r) v[b][r] = cmul(v[b][r], tw[(r - 1) * NS + k]);
             } else {
-                const float2 w1 = Bt[k];
+                const float2 w1 = tw[k];
                 float2 w = w1;
 #pragma unroll
                 for (int r = 1; r < R; ++r) {
@@ -106,20 +119,29 @@ __device__ __forceinline__ void stage(float2 *__restrict__ z, const float2 *__re
         const int k = j & (NS - 1);
         float2 *dst = z + padded((j - k) * R + k);
 #pragma unroll
-        for (int r = 0; r < R; ++r) dst[padded(perm<R>(r) * NS)] = v[b][r];
+        for (int r = 0; r < R; ++r) {
+            dst[padded(perm<R>(r) * NS)] = v[b][r];
+            post((j - k) * R + k + perm<R>(r) * NS, v[b][r]);
+        }
     }
     __syncthreads();
 }
 
-// All stages of one transform; first(index) feeds the first stage unless OWN_FIRST (the column itself).
-template <int LGN, bool OWN_FIRST, typename First>
-__device__ __forceinline__ void transform(float2 *__restrict__ z, const float2 *__restrict__ E, const float2 *__restrict__ Bt, First first) {
+// All stages of one transform.  The first stage reads first(index), or with OWN_FIRST the column itself
+// through pre(value, index); post(index, value) sees the outputs of the last stage.
+template <int LGN, bool OWN_FIRST, typename First, typename Pre, typename Post>
+__device__ __forceinline__ void transform(float2 *__restrict__ z, const float2 *__restrict__ tw2, const float2 *__restrict__ tw3,
+                                          const float2 *__restrict__ chain, First first, Pre pre, Post post) {
     using S = Stages<LGN>;
     constexpr int N = 1 << LGN, NT = threads<LGN>();
-    stage<N, NT, S::R1, 1, OWN_FIRST>(z, E, Bt, first);
-    stage<N, NT, S::R2, S::R1, true>(z, E, Bt, first);
-    if constexpr (S::R3 > 1) stage<N, NT, S::R3, S::R1 * S::R2, true>(z, E, Bt, first);
-    if constexpr (S::R4 > 1) stage<N, NT, S::R4, S::R1 * S::R2 * S::R3, true>(z, E, Bt, first);
+    constexpr int n_stages = S::R4 > 1 ? 4 : (S::R3 > 1 ? 3 : 2);
+    constexpr bool chained3 = n_stages == 3 && tw3_entries<LGN>() == 0;
+    stage<N, NT, S::R1, 1, OWN_FIRST>(z, tw2, first, pre, NoPost());
+    if constexpr (n_stages == 2) stage<N, NT, S::R2, S::R1, true>(z, tw2, first, NoPre(), post);
+    else stage<N, NT, S::R2, S::R1, true>(z, tw2, first, NoPre(), NoPost());
+    if constexpr (n_stages == 3) stage<N, NT, S::R3, S::R1 * S::R2, true>(z, chained3 ? chain : tw3, first, NoPre(), post);
+    else if constexpr (n_stages == 4) stage<N, NT, S::R3, S::R1 * S::R2, true>(z, tw3, first, NoPre(), NoPost());
+    if constexpr (n_stages == 4) stage<N, NT, S::R4, S::R1 * S::R2 * S::R3, true>(z, chain, first, NoPre(), post);
 }
 
 // Block-wide maximum / sum of one value per thread; every thread gets the result.
@@ -170,19 +192,32 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ slot, const int32_t *_
     constexpr int N = 1 << LGN, NT = threads<LGN>(), NC = chain_entries<LGN>();
     extern __shared__ float2 col_smem[];
     __shared__ float red[NT / 32];
+    using S = Stages<LGN>;
+    constexpr int N2 = tw2_entries<LGN>(), N3 = tw3_entries<LGN>();
     float2 *z = col_smem;
-    float2 *E = z + padded(N) + 1;
-    float2 *Bt = E + (1 << kLgE);
+    float2 *tw2 = z + padded(N) + 1;
+    float2 *tw3 = tw2 + N2;
+    float2 *Bt = tw3 + N3;
     const int col = blockIdx.x;
-    for (int i = threadIdx.x; i < (1 << kLgE); i += NT) E[i] = tabE[i];
+    // per-stage twiddle tables, entry (r - 1) * NS + k = e^{+j 2 pi k r / (NS * R)}, from E (first used after barriers)
+    for (int e = threadIdx.x; e < N2; e += NT) {
+        constexpr int NS = S::R1, T = S::R1 * S::R2;
+        tw2[e] = tabE[(e % NS) * (e / NS + 1) * ((1 << kLgE) / T)];
+    }
+    for (int e = threadIdx.x; e < N3; e += NT) {
+        constexpr int NS = S::R1 * S::R2, T = (N3 > 0 ? NS * S::R3 : 1);
+        tw3[e] = tabE[(e % NS) * (e / NS + 1) * ((1 << kLgE) / T)];
+    }
     for (int i = threadIdx.x; i < NC; i += NT) Bt[i] = tabB[i];
     long long tl = (long long)t_len[col / HQ] + t_add;
     if (t_quant > 1 && tl > 0) tl = tl / t_quant * t_quant;      // block-deferred fold: whole blocks only
     const int live = tl < 0 ? 0 : (tl < (long long)P ? (int)tl : (int)P);
     pdl_wait();                                      // Qs comes from the previous kernel
     const float2 *X = Qs + (size_t)col * M;
-    // ---- inverse transform, the half-spectrum packing fused into the first stage's reads
-    transform<LGN, false>(z, E, Bt, [&](int k) {
+    // ---- inverse transform, the half-spectrum packing fused into the first stage's reads; the last stage
+    // leaves z[m] = (s[2m], s[2m+1]) and every thread the maximum of the live scores it wrote
+    float mx = -INFINITY;
+    transform<LGN, false>(z, tw2, tw3, Bt, [&](int k) {
         const int sx = slot[k], sy = slot[N - k];
         float2 v = make_float2(0.f, 0.f);
         if (sx >= 0 || sy >= 0) {
@@ -192,23 +227,20 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ slot, const int32_t *_
             v = cadd(cadd(xk, xm), cmulj(cmul(tabP[k], csub(xk, xm))));
         }
         return v;
-    });
-    // ---- softmax over n < live; z[m] = (s[2m], s[2m+1])
-    float mx = -INFINITY;
-    for (int m = threadIdx.x; m < N; m += NT) {
-        const float2 v = z[padded(m)];
+    }, NoPre(), [&](int m, float2 v) {
         if (2 * m < live) mx = fmaxf(mx, v.x);
         if (2 * m + 1 < live) mx = fmaxf(mx, v.y);
-    }
+    });
     const float m_col = block_reduce<NT, true>(mx, red);
+    // ---- softmax over n < live, applied as the forward transform reads the column:
+    // p[2m] + j p[2m+1] = exp(s - max) on the live positions, 0 elsewhere; then the transform itself
     float sum = 0.f;
-    for (int m = threadIdx.x; m < N; m += NT) {
-        const float2 v = z[padded(m)];
+    transform<LGN, true>(z, tw2, tw3, Bt, [&](int) { return make_float2(0.f, 0.f); }, [&](float2 v, int m) {
         const float pe = 2 * m < live ? __expf(v.x - m_col) : 0.f;
         const float po = 2 * m + 1 < live ? __expf(v.y - m_col) : 0.f;
         sum += pe + po;
-        z[padded(m)] = make_float2(pe, po);
-    }
+        return make_float2(pe, po);
+    }, NoPost());
     const float s_col = block_reduce<NT, false>(sum, red);
     // the window joins the softmax as one more segment: bring both to the joint maximum
     const float mw = m_w != nullptr ? m_w[col] : -INFINITY;
@@ -219,9 +251,6 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ slot, const int32_t *_
         colsum[col] = s_col * f_col + (m_w != nullptr ? s_w[col] * f_w : 0.f);
         colsum[Gp + col] = f_w;
     }
-    __syncthreads();                                 // probabilities in place
-    // ---- forward transform of p[2m] + j p[2m+1]
-    transform<LGN, true>(z, E, Bt, [&](int idx) { return z[padded(idx)]; });
     // ---- unpacking at the retained bins: W[k] = (Zf[k'] + conj Zf[-k'])/2 + e^{+j2pi k/P} (Zf[k'] - conj Zf[-k'])/(2j)
     float2 *out = Wg + (size_t)col * M;
     for (int i = threadIdx.x; i < M; i += NT) {
