@@ -199,6 +199,8 @@ DECODE_WORKLOADS = [
          n_layers=32, n_kv_heads=8, n_q_heads=32, batch=16, T=16384, M=2048),
     dict(name="configs[3]: long context, batch 1, 131072 tokens at 1/16 retention", config=3,
          n_layers=32, n_kv_heads=8, n_q_heads=32, batch=1, T=131072, M=8192),
+    dict(name="configs[4] cell: 32 kv = 32 query heads, batch 32, 4096 tokens at 1/8 retention", config=4,
+         n_layers=32, n_kv_heads=32, n_q_heads=32, batch=32, T=4096, M=512),
 ]
 
 
@@ -641,7 +643,7 @@ def main():
     ap.add_argument("--no-decode-configs", action="store_true",
                     help="skip the decode sections at the configs[2] and configs[3] shapes")
     ap.add_argument("--decode-config-iters", type=int, default=10)
-    ap.add_argument("--only-decode-config", type=int, default=0, choices=[0, 2, 3],
+    ap.add_argument("--only-decode-config", type=int, default=0, choices=[0, 2, 3, 4],
                     help="profiling case: run only the decode section of configs[2] or configs[3] (eager launches; "
                          "combine with --layers and --decode-config-iters 1)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
