@@ -181,27 +181,26 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
 
     __syncthreads();
     pdl_wait();                                      // Y comes from the previous kernel
-    {
-        auto load = [&](int k2, int cidx) {
-            return Y[y_index(g, m1_0 + (cidx >> kLgCW), k2, g0 + (cidx & (kCW - 1)))];
-        };
-        auto store = [&](int m2, int cidx, float2 v) { T[(m2 << lg_cols) + cidx] = v; };
-        fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);      // T[m2][mt, c] = z[m1 + N1 m2]
-    }
-    __syncthreads();
     // a thread always meets the same column: kThreads is a multiple of 16
     const int c = threadIdx.x & (kCW - 1);
     const int live = live_s[c];
     float mx = -INFINITY;
-    for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int mt = (e >> kLgCW) & (MT - 1), m2 = e >> lg_cols;
-        const int n0 = 2 * (m1_0 + mt + g.N1 * m2);
-        const float2 v = T[e];
-        if (n0 < live) mx = fmaxf(mx, v.x);
-        if (n0 + 1 < live) mx = fmaxf(mx, v.y);
+    {
+        auto load = [&](int k2, int cidx) {
+            return Y[y_index(g, m1_0 + (cidx >> kLgCW), k2, g0 + (cidx & (kCW - 1)))];
+        };
+        // T[m2][mt, c] = z[m1 + N1 m2] = scores of positions 2m, 2m + 1; the maximum of the live ones is
+        // collected on the way out of the registers
+        auto store = [&](int m2, int cidx, float2 v) {
+            T[(m2 << lg_cols) + cidx] = v;
+            const int n0 = 2 * (m1_0 + (cidx >> kLgCW) + g.N1 * m2);
+            if (n0 < live) mx = fmaxf(mx, v.x);
+            if (n0 + 1 < live) mx = fmaxf(mx, v.y);
+        };
+        fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
     }
     red[threadIdx.x] = mx;
-    __syncthreads();
+    __syncthreads();                                 // also: the tile is complete
     if (threadIdx.x < kCW) {
         float m = red[threadIdx.x];
 #pragma unroll
@@ -211,31 +210,31 @@ k_afft_mid(fft::Geometry g, float2 *__restrict__ Y, const int32_t *__restrict__ 
     __syncthreads();
     const float mcol = colv[c];
     float sum = 0.f;
-    for (int e = threadIdx.x; e < tile; e += kThreads) {
-        const int mt = (e >> kLgCW) & (MT - 1), m2 = e >> lg_cols;
-        const int n0 = 2 * (m1_0 + mt + g.N1 * m2);
-        const float2 v = T[e];
-        const float pe = n0 < live ? __expf(v.x - mcol) : 0.f;
-        const float po = n0 + 1 < live ? __expf(v.y - mcol) : 0.f;
-        sum += pe + po;
-        T[e] = make_float2(pe, po);
-    }
-    red[threadIdx.x] = sum;
-    __syncthreads();
-    if (threadIdx.x < kCW) {
-        float s = red[threadIdx.x];
-#pragma unroll
-        for (int i = 1; i < kThreads / kCW; ++i) s += red[threadIdx.x + kCW * i];
-        mloc[(size_t)blockIdx.x * g.Gp + g0 + threadIdx.x] = colv[threadIdx.x];
-        sloc[(size_t)blockIdx.x * g.Gp + g0 + threadIdx.x] = s;
-    }
     {
-        auto load = [&](int m2, int cidx) { return T[(m2 << lg_cols) + cidx]; };
+        // p~ = exp(s - tile max) on the live positions, formed as the forward pass reads the tile
+        auto load = [&](int m2, int cidx) {
+            const float2 v = T[(m2 << lg_cols) + cidx];
+            const int n0 = 2 * (m1_0 + (cidx >> kLgCW) + g.N1 * m2);
+            const float pe = n0 < live ? __expf(v.x - mcol) : 0.f;
+            const float po = n0 + 1 < live ? __expf(v.y - mcol) : 0.f;
+            sum += pe + po;
+            return make_float2(pe, po);
+        };
         auto store = [&](int k1p, int cidx, float2 v) {
             const int mt = cidx >> kLgCW;
             Y[y_index(g, m1_0 + mt, k1p, g0 + (cidx & (kCW - 1)))] = cmul(v, tab_i[(k1p << lgMT) + mt]);
         };
         fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
+    }
+    __syncthreads();                                 // red is free again
+    red[threadIdx.x] = sum;
+    __syncthreads();
+    if (threadIdx.x < kCW) {
+        float sm = red[threadIdx.x];
+#pragma unroll
+        for (int i = 1; i < kThreads / kCW; ++i) sm += red[threadIdx.x + kCW * i];
+        mloc[(size_t)blockIdx.x * g.Gp + g0 + threadIdx.x] = colv[threadIdx.x];
+        sloc[(size_t)blockIdx.x * g.Gp + g0 + threadIdx.x] = sm;
     }
 }
 

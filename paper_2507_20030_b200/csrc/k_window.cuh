@@ -202,7 +202,7 @@ inline size_t block_fold_smem(int D) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kFoldWarps * 32, 2)
+__global__ void __launch_bounds__(kFoldWarps * 32, 3)
 k_block_fold(float *__restrict__ coefK, float *__restrict__ coefV, const int32_t *__restrict__ t_len,
              const int32_t *__restrict__ bins, WindowArgs wa, int M, int H, int batch, uint32_t P, int splits) {
     extern __shared__ __align__(16) unsigned char fold_smem[];
