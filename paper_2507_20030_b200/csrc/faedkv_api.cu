@@ -57,6 +57,8 @@ struct FftScratch {
     float2 *colE = nullptr, *colB = nullptr, *colP = nullptr;   // its twiddle tables (see k_col_tables)
     cudaStream_t side = nullptr;          // second stream: the window kernel runs beside the FFT kernels
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaStream_t side2 = nullptr;         // third stream: the second run of sequences of a call cut in two
+    cudaEvent_t ev_cut = nullptr, ev_merge = nullptr;
     unsigned int *tickets = nullptr;      // [max_batch * H + max_batch], zero between calls
     int max_M = 0;
     unsigned int attr_mask[11] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
@@ -169,6 +171,9 @@ void free_scratch(faedkv_ctx *ctx) {
     if (f.side != nullptr) cudaStreamDestroy(f.side);
     if (f.ev_fork != nullptr) cudaEventDestroy(f.ev_fork);
     if (f.ev_join != nullptr) cudaEventDestroy(f.ev_join);
+    if (f.side2 != nullptr) cudaStreamDestroy(f.side2);
+    if (f.ev_cut != nullptr) cudaEventDestroy(f.ev_cut);
+    if (f.ev_merge != nullptr) cudaEventDestroy(f.ev_merge);
     f = FftScratch();
 }
 
@@ -237,6 +242,9 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             CUDA_TRY(ctx, cudaMalloc(&f.colE, sizeof(float2) << colfft::kLgE));
             CUDA_TRY(ctx, cudaMalloc(&f.colB, sizeof(float2) << colfft::kLgE));
             CUDA_TRY(ctx, cudaMalloc(&f.colP, sizeof(float2) * ((size_t)g.N + 1)));
+            CUDA_TRY(ctx, cudaStreamCreateWithFlags(&f.side2, cudaStreamNonBlocking));
+            CUDA_TRY(ctx, cudaEventCreateWithFlags(&f.ev_cut, cudaEventDisableTiming));
+            CUDA_TRY(ctx, cudaEventCreateWithFlags(&f.ev_merge, cudaEventDisableTiming));
             colfft::k_col_tables<<<32, 256>>>(f.colE, f.colB, f.colP, (uint32_t)c.n_dft);
             CUDA_TRY(ctx, cudaDeviceSynchronize());
         }
@@ -597,6 +605,19 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
     const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks));
     const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks));
     constexpr int KB = 16 / GQ;
+    // step (5) for the sequences [b0, b1) on stream s
+    auto launch_out = [&](int b0, int b1, cudaStream_t s) -> int {
+        const int nb = b1 - b0;
+        const int slices = out_slices(ctx, nb, M);
+        const int per = (M + slices - 1) / slices;
+        dim3 grid(slices, nb * H);
+        launch_pdl(k_attn_out_fft<TQ, GQ, APPEND>, grid, dim3(kAttnWarps * 32), 0, s,
+                   coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
+                   static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, counts_new ? 1 : 0,
+                   windowed ? WindowArgs{winK, winV, k_new, v_new, S, R, D, Rc, 0.f, nullptr, nullptr, nullptr} : WindowArgs{},
+                   ctx->use_col ? f.Wg : nullptr, b0 * H, batch * H);
+        return launch_check(ctx, "k_attn_out_fft");
+    };
     if (n_extra) {
         // the window's scores, statistics (one more "tile" row) and unnormalised output depend on nothing this call
         // computes: they run on the context's second stream from the top of the call, beside the pass over
@@ -623,26 +644,49 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         if (n_extra) CUDA_TRY(ctx, cudaStreamWaitEvent(st, f.ev_join, 0));
         const int n_tiles = g.N1 >> lgMT;
         const float *m_w = n_extra ? f.mloc + (size_t)n_tiles * g.Gp : nullptr, *s_w = n_extra ? f.sloc + (size_t)n_tiles * g.Gp : nullptr;
+        // With more columns than the GPU holds at once (two CTAs per SM) the last wave of the column kernel leaves
+        // SMs idle and the whole kernel leaves DRAM idle: the batch is then cut into two runs of sequences, each
+        // with its own column kernel and pass over C_V, the second on another stream, so that the first run's
+        // pass over C_V streams while the second run's columns are still being transformed.
+        const int b_cut = (batch >= 2 && batch * HQ > 2 * 148) ? batch / 2 : batch;
+        auto launch_col = [&](int b0, int b1, cudaStream_t s) -> int {
+            int rcc = FAEDKV_ERR_UNSUPPORTED;
 #define CALL(LG)                                                                                         \
-        rc = fft_opt_in(ctx, colfft::k_afft_col<LG>, colfft::smem_bytes<LG>(), f.attr_mask[10], LG);      \
-        if (rc == 0) launch_pdl(colfft::k_afft_col<LG>, dim3(batch * HQ), dim3(colfft::threads<LG>()), colfft::smem_bytes<LG>(), st, \
-                                (uint32_t)P, M, p.d_slot, p.d_bins, f.Qs, f.colE, f.colB, f.colP, t_len, HQ,        \
-                                (counts_new ? 1 : 0) - S - R, D, m_w, s_w, f.Wg, f.colsum, g.Gp)
-        switch (g.lgN1 + g.lgN2) {
-            case 5: CALL(5); break;
-            case 6: CALL(6); break;
-            case 7: CALL(7); break;
-            case 8: CALL(8); break;
-            case 9: CALL(9); break;
-            case 10: CALL(10); break;
-            case 11: CALL(11); break;
-            case 12: CALL(12); break;
-            case 13: CALL(13); break;
-            default: break;
-        }
+            rcc = fft_opt_in(ctx, colfft::k_afft_col<LG>, colfft::smem_bytes<LG>(), f.attr_mask[10], LG);  \
+            if (rcc == 0) launch_pdl(colfft::k_afft_col<LG>, dim3((b1 - b0) * HQ), dim3(colfft::threads<LG>()), colfft::smem_bytes<LG>(), s, \
+                                     (uint32_t)P, M, p.d_slot, p.d_bins, f.Qs, f.colE, f.colB, f.colP, t_len, HQ,   \
+                                     (counts_new ? 1 : 0) - S - R, D, m_w, s_w, f.Wg, f.colsum, g.Gp, b0 * HQ)
+            switch (g.lgN1 + g.lgN2) {
+                case 5: CALL(5); break;
+                case 6: CALL(6); break;
+                case 7: CALL(7); break;
+                case 8: CALL(8); break;
+                case 9: CALL(9); break;
+                case 10: CALL(10); break;
+                case 11: CALL(11); break;
+                case 12: CALL(12); break;
+                case 13: CALL(13); break;
+                default: break;
+            }
 #undef CALL
-        if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no column kernel for 2^%d points", g.lgN1 + g.lgN2) : rc;
-        if (int r = launch_check(ctx, "k_afft_col")) return r;
+            if (rcc) return rcc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rcc, "no column kernel for 2^%d points", g.lgN1 + g.lgN2) : rcc;
+            return launch_check(ctx, "k_afft_col");
+        };
+        if (b_cut < batch) {
+            CUDA_TRY(ctx, cudaEventRecord(f.ev_cut, st));
+            CUDA_TRY(ctx, cudaStreamWaitEvent(f.side2, f.ev_cut, 0));
+        }
+        if (int r = launch_col(0, b_cut, st)) return r;
+        if (b_cut < batch) {
+            if (int r = launch_col(b_cut, batch, f.side2)) return r;
+        }
+        if (int r = launch_out(0, b_cut, st)) return r;
+        if (b_cut < batch) {
+            if (int r = launch_out(b_cut, batch, f.side2)) return r;
+            CUDA_TRY(ctx, cudaEventRecord(f.ev_merge, f.side2));
+            CUDA_TRY(ctx, cudaStreamWaitEvent(st, f.ev_merge, 0));
+        }
+        rc = FAEDKV_OK;
     } else {
     rc = FAEDKV_ERR_UNSUPPORTED;
     {
@@ -682,16 +726,8 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         if (int r = launch_check(ctx, "k_afft_fwd_b")) return r;
     }
     }
-    {
-        const int slices = out_slices(ctx, batch, M);
-        const int per = (M + slices - 1) / slices;
-        dim3 grid(slices, batch * H);
-        launch_pdl(k_attn_out_fft<TQ, GQ, APPEND>, grid, dim3(kAttnWarps * 32), 0, st,
-                   coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
-                   static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, counts_new ? 1 : 0,
-                   windowed ? WindowArgs{winK, winV, k_new, v_new, S, R, D, Rc, 0.f, nullptr, nullptr, nullptr} : WindowArgs{},
-                   ctx->use_col ? f.Wg : nullptr);
-        if (int r = launch_check(ctx, "k_attn_out_fft")) return r;
+    if (!ctx->use_col) {
+        if (int r = launch_out(0, batch, st)) return r;
     }
     return FAEDKV_OK;
 }

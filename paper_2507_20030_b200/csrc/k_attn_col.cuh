@@ -187,7 +187,7 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ slot, const int32_t *_
            const float2 *__restrict__ Qs, const float2 *__restrict__ tabE, const float2 *__restrict__ tabB,
            const float2 *__restrict__ tabP, const int32_t *__restrict__ t_len, int HQ, int t_add, int t_quant,
            const float *__restrict__ m_w, const float *__restrict__ s_w, float2 *__restrict__ Wg,
-           float *__restrict__ colsum, int Gp) {
+           float *__restrict__ colsum, int Gp, int col0) {
     using namespace fft;
     constexpr int N = 1 << LGN, NT = threads<LGN>(), NC = chain_entries<LGN>();
     extern __shared__ float2 col_smem[];
@@ -198,7 +198,7 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ slot, const int32_t *_
     float2 *tw2 = z + padded(N) + 1;
     float2 *tw3 = tw2 + N2;
     float2 *Bt = tw3 + N3;
-    const int col = blockIdx.x;
+    const int col = col0 + (int)blockIdx.x;          // a launch may cover a run of columns
     // per-stage twiddle tables, entry (r - 1) * NS + k = e^{+j 2 pi k r / (NS * R)}, from E (first used after barriers)
     for (int e = threadIdx.x; e < N2; e += NT) {
         constexpr int NS = S::R1, T = S::R1 * S::R2;

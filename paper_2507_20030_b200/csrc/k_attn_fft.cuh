@@ -346,7 +346,8 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
                const float2 *__restrict__ Zf, const float *__restrict__ colsum, const int32_t *__restrict__ bins,
                float *__restrict__ partial, unsigned int *__restrict__ tickets, TQ *__restrict__ out,
                int M, int H, int HQ, fft::Geometry g, int bins_per_slice, float inv_P, FoldSrc fold,
-               const float *__restrict__ o_win, int bump, WindowArgs commit, const float2 *__restrict__ Wg) {
+               const float *__restrict__ o_win, int bump, WindowArgs commit, const float2 *__restrict__ Wg,
+               int bh0, int n_units) {
     using namespace fft;
     // the weights of a chunk and the final cross-warp reduction share one buffer
     constexpr size_t kWgtBytes = (size_t)kOutChunk * GQ * sizeof(float2) + (APPEND ? kOutChunk * sizeof(float2) : 0);
@@ -357,7 +358,8 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
     float (*red)[GQ][kHeadDim] = reinterpret_cast<float (*)[GQ][kHeadDim]>(sbuf);
     __shared__ unsigned int last_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bh = blockIdx.y, b = bh / H, h = bh % H;
+    // a launch may cover a run of whole sequences only: units [bh0, bh0 + gridDim.y) of n_units
+    const int bh = bh0 + (int)blockIdx.y, b = bh / H, h = bh % H;
     const int kbeg = blockIdx.x * bins_per_slice;
     const int kend = min(M, kbeg + bins_per_slice);
     const size_t plane = (size_t)M * kHeadDim;
@@ -482,9 +484,9 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
             // its ring slot (windowed step) and advances the counter
             __shared__ unsigned int seq_last;
             if (threadIdx.x == 0) {
-                const unsigned int done = atomicAdd(&tickets[gridDim.y + b], 1u);
+                const unsigned int done = atomicAdd(&tickets[n_units + b], 1u);
                 seq_last = done == (unsigned int)H - 1u ? 1u : 0u;
-                if (seq_last) tickets[gridDim.y + b] = 0u;
+                if (seq_last) tickets[n_units + b] = 0u;
             }
             __syncthreads();
             if (seq_last) {

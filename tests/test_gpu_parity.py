@@ -287,6 +287,9 @@ def _decode_modes(fk, dtype, P):
     # grid (relative 2^-9) stays finer than the absolute tolerance.
     (64, 64, 33, 1, 2, 4, [33], 0.125),
     (4096, 4096, 96, 3, 2, 8, [4096, 1, 2049], 0.125),   # two-pass split 64 x 32; a one-token sequence
+    # 320 columns: more than the GPU holds at once, so the column-transform path cuts the batch into two
+    # runs of sequences (2 + 3) on two streams; ragged lengths
+    (128, 128, 20, 5, 8, 64, [128, 9, 77, 128, 30], 0.125),
 ])
 def test_decode_attn_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, tl, vscale):
     from paper_2507_20030_b200 import synth
