@@ -71,7 +71,8 @@ def test_create_rejects_bad_configs_before_touching_cuda(lib):
                 kv_dtype=binding.F32, prefill_mode=0, twiddle_terms=0, decode_mode=0)
     for key, bad, code in [("head_dim", 64, -4), ("n_dft", 1, -1), ("n_q_heads", 12, -4),
                            ("n_q_heads", 128, -4), ("kv_dtype", 7, -1), ("max_batch", 0, -1),
-                           ("twiddle_terms", 3, -1), ("n_layers", 0, -1), ("decode_mode", 5, -1)]:
+                           ("twiddle_terms", 3, -1), ("n_layers", 0, -1), ("decode_mode", 5, -1),
+                           ("n_defer", -1, -1), ("n_defer", 129, -1), ("n_sink", 2000, -1)]:
         cfg = binding.Config(**{**good, key: bad})
         assert lib.faedkv_create(ctypes.byref(cfg), ctypes.byref(h)) == code, key
         assert not h.value
