@@ -334,7 +334,7 @@ def test_decode_attn_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, tl, vs
 
 
 @pytest.mark.parametrize("P,M,B,H,HQ", [(32768, 48, 1, 2, 8), (131072, 32, 2, 1, 4), (16384, 64, 3, 2, 4),
-                                         (8192, 64, 2, 2, 2), (4096, 32, 2, 1, 8)])
+                                         (8192, 64, 2, 2, 2), (4096, 32, 2, 1, 8), (65536, 32, 1, 2, 4), (262144, 32, 1, 1, 2)])
 def test_decode_attn_fft_long_grids(fk, oracle, P, M, B, H, HQ):
     """FFT-shaped transforms at the grid sizes of the long-context workloads (few bins, so that the
     oracle's materialised reconstruction stays cheap); ragged live lengths."""
