@@ -644,11 +644,13 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         if (n_extra) CUDA_TRY(ctx, cudaStreamWaitEvent(st, f.ev_join, 0));
         const int n_tiles = g.N1 >> lgMT;
         const float *m_w = n_extra ? f.mloc + (size_t)n_tiles * g.Gp : nullptr, *s_w = n_extra ? f.sloc + (size_t)n_tiles * g.Gp : nullptr;
-        // With more columns than the GPU holds at once (two CTAs per SM) the last wave of the column kernel leaves
+        // With more columns than the GPU holds at once (two CTAs per SM at 8192 points) the last wave of the column kernel leaves
         // SMs idle and the whole kernel leaves DRAM idle: the batch is then cut into two runs of sequences, each
         // with its own column kernel and pass over C_V, the second on another stream, so that the first run's
         // pass over C_V streams while the second run's columns are still being transformed.
-        const int b_cut = (batch >= 2 && batch * HQ > 2 * 148) ? batch / 2 : batch;
+        const int lgn = g.lgN1 + g.lgN2;
+        const int ctas_per_sm = lgn >= 13 ? 2 : (lgn == 12 ? 3 : (lgn == 11 ? 7 : 16));   // registers / shared memory
+        const int b_cut = (batch >= 2 && batch * HQ > ctas_per_sm * 148) ? batch / 2 : batch;
         auto launch_col = [&](int b0, int b1, cudaStream_t s) -> int {
             int rcc = FAEDKV_ERR_UNSUPPORTED;
 #define CALL(LG)                                                                                         \
