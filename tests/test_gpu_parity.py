@@ -533,13 +533,16 @@ def test_prefill_fft_matches_oracle(fk, oracle, dtype, P, T, M, B, H):
     (64, 30, 9, 1, 2, 4, 6, 0, 6),            # no ring: the new token itself is folded
     (1024, 60, 24, 2, 2, 4, 10, 50, 4),       # T = S + R: the transformed segment starts empty
 ])
-def test_windowed_step_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, S, R, steps):
+@pytest.mark.parametrize("two_pass", [False, True])
+def test_windowed_step_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, S, R, steps, two_pass):
     """Prefill with sink + recent window, then decode steps: attention outputs, planes, window contents
-    and counters against the oracle's WindowedUnit, unit by unit."""
+    and counters against the oracle's WindowedUnit, unit by unit; through the one-kernel column transform
+    and through the two-pass transform kernels."""
     from paper_2507_20030_b200 import synth
     GQ = HQ // H
     ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
-                     prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R)
+                     prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R,
+                     decode_mode=fk.DECODE_FFT_TWO_PASS if two_pass else fk.DECODE_AUTO)
     mask = _random_mask(P, M, 13 * P + T)
     mask[0] = 1
     M = int(mask.sum())
@@ -590,14 +593,16 @@ def test_windowed_step_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, S, R
     (64, (20, 21), 9, 1, 1, 0, 0, 2, 7),           # no window at all: nothing waits at a block boundary
     (1024, (60,), 24, 2, 4, 10, 50, 128, 140),     # T = S + R: the planes start empty; the largest block
 ])
-def test_deferred_step_matches_oracle(fk, oracle, dtype, P, Ts, M, H, HQ, S, R, D, steps):
+@pytest.mark.parametrize("two_pass", [False, True])
+def test_deferred_step_matches_oracle(fk, oracle, dtype, P, Ts, M, H, HQ, S, R, D, steps, two_pass):
     """Block-deferred fold: prefill (one call per sequence, so that the batch is ragged), then decode steps
     over the whole batch: attention outputs at every step, final planes, ring contents and counters against
     the oracle's WindowedUnit(defer=D), unit by unit."""
     from paper_2507_20030_b200 import synth
     B, GQ = len(Ts), HQ // H
     ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
-                     prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R, n_defer=D)
+                     prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R, n_defer=D,
+                     decode_mode=fk.DECODE_FFT_TWO_PASS if two_pass else fk.DECODE_AUTO)
     mask = _random_mask(P, M, 17 * P + Ts[0])
     mask[0] = 1
     ctx.plan(0, mask)
