@@ -656,7 +656,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
 #define CALL(LG)                                                                                         \
             rcc = fft_opt_in(ctx, colfft::k_afft_col<LG>, colfft::smem_bytes<LG>(), f.attr_mask[10], LG);  \
             if (rcc == 0) launch_pdl(colfft::k_afft_col<LG>, dim3((b1 - b0) * HQ), dim3(colfft::threads<LG>()), colfft::smem_bytes<LG>(), s, \
-                                     (uint32_t)P, M, p.d_slot, p.d_bins, f.Qs, f.colE, f.colB, f.colP, t_len, HQ,   \
+                                     (uint32_t)P, M, p.d_bins, f.Qs, f.colE, f.colB, f.colP, t_len, HQ,   \
                                      (counts_new ? 1 : 0) - S - R, D, m_w, s_w, f.Wg, f.colsum, g.Gp, b0 * HQ)
             switch (g.lgN1 + g.lgN2) {
                 case 5: CALL(5); break;

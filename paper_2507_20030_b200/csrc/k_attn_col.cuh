@@ -3,7 +3,7 @@
 // transform of the score spectrum, the softmax over the live positions and the forward transform of the
 // probabilities (Eq. 3 on Eq. 11, same packing and unpacking formulas as k_fft.cuh) run without leaving it:
 //
-//   gather     Z[k] from the retained bins of Qs (half-spectrum packing), read by the first butterfly stage
+//   pack       Z[k] from the retained bins of Qs (half-spectrum packing), scattered into the zeroed column
 //   inverse    z[m] = s[2m] + j s[2m+1]: in-place Stockham stages of radix 4 / 8 / 16 over the whole column
 //   softmax    maximum and sum over n < live, p = exp(s - max), in place; the sink + recent window, when there
 //              is one, joins here (its statistics come from k_attn_window)
@@ -175,7 +175,7 @@ __global__ void k_col_tables(float2 *__restrict__ E, float2 *__restrict__ Bt, fl
 }
 
 // Qs: [G][M] (column-major: a column's retained score spectrum is contiguous), already scaled by
-// scale / P, imaginary part of the self-conjugate bins zero.  slot: [N + 1] bin -> index in the plan or -1.
+// scale / P, imaginary part of the self-conjugate bins zero.  bins: [M] the plan's retained bins, ascending.
 // live length of a column = min(q(t_len[col / HQ] + t_add), P), q() rounding down to a multiple of t_quant.
 // m_w, s_w: statistics of the window tile ([G] each) or nullptr.  Out: Wg [G][M] = (w Re Pf, -w Im Pf),
 // scaled to the joint maximum; colsum[col] = joint softmax normaliser, colsum[Gp + col] = the factor that
@@ -183,7 +183,7 @@ __global__ void k_col_tables(float2 *__restrict__ E, float2 *__restrict__ Bt, fl
 // grid = (G); block = threads<LGN>(); dynamic smem = smem_bytes<LGN>().
 template <int LGN>
 __global__ void __launch_bounds__(threads<LGN>(), threads<LGN>() >= 512 ? 2 : 1)
-k_afft_col(uint32_t P, int M, const int32_t *__restrict__ slot, const int32_t *__restrict__ bins,
+k_afft_col(uint32_t P, int M, const int32_t *__restrict__ bins,
            const float2 *__restrict__ Qs, const float2 *__restrict__ tabE, const float2 *__restrict__ tabB,
            const float2 *__restrict__ tabP, const int32_t *__restrict__ t_len, int HQ, int t_add, int t_quant,
            const float *__restrict__ m_w, const float *__restrict__ s_w, float2 *__restrict__ Wg,
@@ -214,20 +214,36 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ slot, const int32_t *_
     const int live = tl < 0 ? 0 : (tl < (long long)P ? (int)tl : (int)P);
     pdl_wait();                                      // Qs comes from the previous kernel
     const float2 *X = Qs + (size_t)col * M;
-    // ---- inverse transform, the half-spectrum packing fused into the first stage's reads; the last stage
-    // leaves z[m] = (s[2m], s[2m+1]) and every thread the maximum of the live scores it wrote
-    float mx = -INFINITY;
-    transform<LGN, false>(z, tw2, tw3, Bt, [&](int k) {
-        const int sx = slot[k], sy = slot[N - k];
-        float2 v = make_float2(0.f, 0.f);
-        if (sx >= 0 || sy >= 0) {
-            const float2 xk = sx >= 0 ? X[sx] : make_float2(0.f, 0.f);
-            float2 xm = sy >= 0 ? X[sy] : make_float2(0.f, 0.f);
-            xm.y = -xm.y;                            // conj X[N-k]
-            v = cadd(cadd(xk, xm), cmulj(cmul(tabP[k], csub(xk, xm))));
+    // ---- half-spectrum packing, from the retained bins outwards (most of the N points are zero):
+    //   Z[k] = X[k] (1 + j e^{+j2pi k/P}) + conj(X[N-k]) (1 - j e^{+j2pi k/P})
+    // every retained bin b < N lands on point b, every retained bin b > 0 on point N - b; a point gets at most
+    // one term of each kind, so two rounds of plain stores / read-modify-writes need no atomics
+    for (int i = threadIdx.x; i < N; i += NT) z[padded(i)] = make_float2(0.f, 0.f);
+    __syncthreads();
+    for (int i = threadIdx.x; i < M; i += NT) {
+        const int bin = bins[i];
+        if (bin < N) {
+            const float2 ph = tabP[bin];
+            z[padded(bin)] = cmul(X[i], make_float2(1.f - ph.y, ph.x));          // 1 + j ph
         }
-        return v;
-    }, NoPre(), [&](int m, float2 v) {
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < M; i += NT) {
+        const int bin = bins[i];
+        if (bin > 0) {
+            const int k = N - bin;
+            const float2 ph = tabP[k];
+            const float2 x = X[i];
+            const float2 t = cmul(make_float2(x.x, -x.y), make_float2(1.f + ph.y, -ph.x));   // conj(X) (1 - j ph)
+            float2 &dst = z[padded(k)];
+            dst = cadd(dst, t);
+        }
+    }
+    __syncthreads();
+    // ---- inverse transform in place; the last stage leaves z[m] = (s[2m], s[2m+1]) and every thread the
+    // maximum of the live scores it wrote
+    float mx = -INFINITY;
+    transform<LGN, true>(z, tw2, tw3, Bt, [&](int) { return make_float2(0.f, 0.f); }, NoPre(), [&](int m, float2 v) {
         if (2 * m < live) mx = fmaxf(mx, v.x);
         if (2 * m + 1 < live) mx = fmaxf(mx, v.y);
     });
