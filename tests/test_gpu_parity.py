@@ -333,6 +333,41 @@ def test_decode_attn_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, tl, vs
         ctx.close()
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_decode_attn_random_shapes(fk, oracle, seed):
+    """Seeded random shapes over every column length the one-kernel transform is instantiated for
+    (P = 64 ... 16384), random retained sets, GQA factors, batch sizes and ragged live lengths (random
+    coefficient planes with a decaying spectrum, so that the oracle's materialised form stays cheap):
+    default mode and the two-pass kernels against the oracle."""
+    from paper_2507_20030_b200 import synth
+    rng = np.random.default_rng(1000 + seed)
+    P = 1 << int(rng.integers(6, 15))
+    GQ = int(rng.choice([1, 2, 4, 8]))
+    H = int(rng.integers(1, 4))
+    B = int(rng.integers(1, 4))
+    M = int(rng.integers(1, min(P // 2 + 1, 96) + 1))
+    HQ = H * GQ
+    mask = _random_mask(P, M, seed)
+    bins = oracle.plan(P, mask)
+    amp = np.sqrt(P) * np.exp(-np.arange(M) / max(M / 3.0, 1.0))[None, None, None, :, None]
+    cK = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * amp).astype(np.float32)).cuda()
+    cV = torch.from_numpy((rng.standard_normal((B, H, 2, M, 128)) * amp).astype(np.float32)).cuda()
+    tl = rng.integers(1, 2 * P, size=B).astype(np.int32)          # some beyond P: live length is capped
+    t_len = torch.from_numpy(tl).cuda()
+    q = synth.make_q(seed, 0, B, HQ, 128, dtype=torch.float32)
+    want = oracle_decode_attn(oracle, q, to_np64(cK), to_np64(cV), P, bins, tl)
+    for mode in (fk.DECODE_AUTO, fk.DECODE_FFT_TWO_PASS):
+        ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=fk.F32, decode_mode=mode)
+        ctx.plan(0, mask)
+        out = torch.full((B, HQ, 128), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.decode_attn(0, q.cuda(), cK, cV, t_len, out)
+        torch.cuda.synchronize()
+        err = np.abs(to_np64(out) - want).max()
+        assert err <= ATTN_MAX_ABS, (seed, P, M, B, H, GQ, mode, err)
+        assert ctx.device_status() == 0
+        ctx.close()
+
+
 @pytest.mark.parametrize("P,M,B,H,HQ", [(32768, 48, 1, 2, 8), (131072, 32, 2, 1, 4), (16384, 64, 3, 2, 4),
                                          (8192, 64, 2, 2, 2), (4096, 32, 2, 1, 8), (65536, 32, 1, 2, 4), (262144, 32, 1, 1, 2)])
 def test_decode_attn_fft_long_grids(fk, oracle, P, M, B, H, HQ):
