@@ -369,7 +369,8 @@ def test_decode_attn_random_shapes(fk, oracle, seed):
 
 
 @pytest.mark.parametrize("P,M,B,H,HQ", [(32768, 48, 1, 2, 8), (131072, 32, 2, 1, 4), (16384, 64, 3, 2, 4),
-                                         (8192, 64, 2, 2, 2), (4096, 32, 2, 1, 8), (65536, 32, 1, 2, 4), (262144, 32, 1, 1, 2)])
+                                         (8192, 64, 2, 2, 2), (4096, 32, 2, 1, 8), (65536, 32, 1, 2, 4), (262144, 32, 1, 1, 2),
+                                         (524288, 32, 1, 1, 1)])       # the largest grid the FFT-shaped path takes
 def test_decode_attn_fft_long_grids(fk, oracle, P, M, B, H, HQ):
     """FFT-shaped transforms at the grid sizes of the long-context workloads (few bins, so that the
     oracle's materialised reconstruction stays cheap); ragged live lengths."""

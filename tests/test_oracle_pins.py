@@ -398,6 +398,47 @@ def test_mixed_mask_independent_restatement(oracle):
     np.testing.assert_array_equal(got, want)
 
 
+# ----------------------------------------------------------------------------- structural identities
+def test_shift_theorem_and_linearity(oracle):
+    """Delaying the sequence by d positions multiplies bin k by e^{-j2 pi k d / P} (the `pos0` argument is
+    that delay), and the transform is linear: two facts a wrong phase sign, a transposed index or a
+    dropped term in the pruned DFT cannot satisfy together."""
+    P, T, d = 48, 31, 5
+    rng = np.random.default_rng(77)
+    x, y = rng.standard_normal((T, d)), rng.standard_normal((T, d))
+    mask = np.zeros(P // 2 + 1, dtype=np.uint8)
+    mask[[0, 1, 4, 9, 17, 24]] = 1
+    bins = oracle.plan(P, mask)
+    cx = np.array(oracle.compress(x, P, bins))
+    cy = np.array(oracle.compress(y, P, bins))
+    cz = np.array(oracle.compress(2.5 * x - 0.75 * y, P, bins))
+    assert np.abs(cz - (2.5 * cx - 0.75 * cy)).max() < 1e-11
+    for delay in (1, 7, P - 3, P + 2):
+        sh = np.array(oracle.compress(x, P, bins, pos0=delay))
+        ph = np.exp(-2j * np.pi * bins * delay / P)[:, None]
+        want = (cx[0] + 1j * cx[1]) * ph
+        assert np.abs(sh[0] + 1j * sh[1] - want).max() < 1e-10, delay
+
+
+def test_reconstruction_is_the_best_band_limited_fit(oracle):
+    """Eq. 5 on the retained bins of Eq. 4 is the orthogonal projection of the (zero-padded) sequence onto
+    those frequencies: the residual is orthogonal to every retained cosine and sine, and no other
+    coefficient vector on the same bins fits better (numpy least squares on the real basis)."""
+    P, d = 40, 3
+    rng = np.random.default_rng(78)
+    x = rng.standard_normal((P, d))
+    mask = np.zeros(P // 2 + 1, dtype=np.uint8)
+    mask[[0, 2, 3, 11, 20]] = 1
+    bins = oracle.plan(P, mask)
+    re, im = oracle.compress(x, P, bins)
+    rec = oracle.reconstruct(re, im, P, bins, P)
+    n = np.arange(P)[:, None]
+    basis = np.concatenate([np.cos(2 * np.pi * n * bins[None, :] / P), np.sin(2 * np.pi * n * bins[None, :] / P)], axis=1)
+    assert np.abs(basis.T @ (x - rec)).max() < 1e-10
+    fit = basis @ np.linalg.lstsq(basis, x, rcond=None)[0]
+    assert np.abs(fit - rec).max() < 1e-10
+
+
 # ----------------------------------------------------------------------------- sink + recent window
 def _numpy_attention(q, K, V, scale):
     s = (q @ K.T) * scale
