@@ -24,7 +24,7 @@ namespace faedkv {
 // ---- (1) ------------------------------------------------------------------------------------------
 // grid = (ceil(M / (8 * KB)), batch * H); block = 256; KB = 16 / GQ bins per warp.
 template <typename TQ, int GQ, bool APPEND>
-__global__ void __launch_bounds__(kAttnWarps * 32)
+__global__ void __launch_bounds__(kAttnWarps * 32, 3)
 k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restrict__ k_new,
           const int32_t *__restrict__ t_len, const int32_t *__restrict__ bins, float2 *__restrict__ Qs,
           int M, int H, int HQ, int Gp, uint32_t P, float scale_over_P, FoldSrc fold, int col_major) {
@@ -39,46 +39,56 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
     for (int g = 0; g < GQ; ++g) qv[g] = load4(q + ((size_t)b * HQ + h * GQ + g) * kHeadDim + lane * 4);
     const size_t plane = (size_t)M * kHeadDim;
     float *base = coefK + (size_t)bh * 2 * plane;
-    float4 row[KB][2];
-#pragma unroll
-    for (int kk = 0; kk < KB; ++kk)
-#pragma unroll
-        for (int pl = 0; pl < 2; ++pl) {
-            row[kk][pl] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (k0 + kk < M) row[kk][pl] = ld_stream(base + pl * plane + (size_t)(k0 + kk) * kHeadDim + lane * 4);
-        }
+    // C_K[k, c] += x[c] * e^{-j w k t} (APPEND): same arithmetic as k_append; x is the call's new token, or with a
+    // recent window the token that leaves it (k_new then points at the window tensor)
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    uint32_t t = 0;
     if (APPEND) {
-        // C_K[k, c] += x[c] * e^{-j w k t}: same arithmetic as k_append; x is the call's new token, or with a
-        // recent window the token that leaves it (k_new then points at the window tensor)
         size_t xrow;
-        uint32_t t;
         fold_locate(fold, t_len[b], bh, P, xrow, t);
-        const float4 x = load4(k_new + xrow * kHeadDim + lane * 4);
-#pragma unroll
-        for (int kk = 0; kk < KB; ++kk) {
-            if (k0 + kk >= M) continue;
-            float c, s;
-            twiddle(phase_mod((uint32_t)bins[k0 + kk], t, P), P, c, s);
-            float4 &re = row[kk][0], &im = row[kk][1];
-            re.x = fmaf(x.x, c, re.x); im.x = fmaf(-x.x, s, im.x);
-            re.y = fmaf(x.y, c, re.y); im.y = fmaf(-x.y, s, im.y);
-            re.z = fmaf(x.z, c, re.z); im.z = fmaf(-x.z, s, im.z);
-            re.w = fmaf(x.w, c, re.w); im.w = fmaf(-x.w, s, im.w);
-            float *dst = base + (size_t)(k0 + kk) * kHeadDim + lane * 4;
-            st_stream(dst, re);
-            st_stream(dst + plane, im);
-        }
+        x = load4(k_new + xrow * kHeadDim + lane * 4);
     }
+    // The warp's KB bins go through in groups of at most 4: rows of a group are loaded together, updated and
+    // written back (APPEND), reduced to their dot products, and only those stay live.  (All 16 bins of the
+    // one-query-head case at once took 158 registers with the update fused: one CTA per SM, 3.9 TB/s.)
+    constexpr int GB = KB < 4 ? KB : 4;
     float v[32];
 #pragma unroll
-    for (int kk = 0; kk < KB; ++kk)
+    for (int g0 = 0; g0 < KB; g0 += GB) {
+        float4 row[GB][2];
 #pragma unroll
-        for (int pl = 0; pl < 2; ++pl)
+        for (int kk = 0; kk < GB; ++kk)
 #pragma unroll
-            for (int g = 0; g < GQ; ++g) {
-                const float4 r = row[kk][pl];
-                v[(kk * 2 + pl) * GQ + g] = r.x * qv[g].x + r.y * qv[g].y + r.z * qv[g].z + r.w * qv[g].w;
+            for (int pl = 0; pl < 2; ++pl) {
+                row[kk][pl] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (k0 + g0 + kk < M) row[kk][pl] = ld_stream(base + pl * plane + (size_t)(k0 + g0 + kk) * kHeadDim + lane * 4);
             }
+        if (APPEND) {
+#pragma unroll
+            for (int kk = 0; kk < GB; ++kk) {
+                if (k0 + g0 + kk >= M) continue;
+                float c, sn;
+                twiddle(phase_mod((uint32_t)bins[k0 + g0 + kk], t, P), P, c, sn);
+                float4 &re = row[kk][0], &im = row[kk][1];
+                re.x = fmaf(x.x, c, re.x); im.x = fmaf(-x.x, sn, im.x);
+                re.y = fmaf(x.y, c, re.y); im.y = fmaf(-x.y, sn, im.y);
+                re.z = fmaf(x.z, c, re.z); im.z = fmaf(-x.z, sn, im.z);
+                re.w = fmaf(x.w, c, re.w); im.w = fmaf(-x.w, sn, im.w);
+                float *dst = base + (size_t)(k0 + g0 + kk) * kHeadDim + lane * 4;
+                st_stream(dst, re);
+                st_stream(dst + plane, im);
+            }
+        }
+#pragma unroll
+        for (int kk = 0; kk < GB; ++kk)
+#pragma unroll
+            for (int pl = 0; pl < 2; ++pl)
+#pragma unroll
+                for (int g = 0; g < GQ; ++g) {
+                    const float4 r = row[kk][pl];
+                    v[((g0 + kk) * 2 + pl) * GQ + g] = r.x * qv[g].x + r.y * qv[g].y + r.z * qv[g].z + r.w * qv[g].w;
+                }
+    }
     const float tot = warp_transpose_reduce32(v, lane);
     const int kk = lane / (2 * GQ), pl = (lane / GQ) & 1, g = lane % GQ;
     if (k0 + kk < M) {
