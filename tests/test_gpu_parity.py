@@ -690,6 +690,64 @@ def test_deferred_step_matches_oracle(fk, oracle, dtype, P, Ts, M, H, HQ, S, R, 
     ctx.close()
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_windowed_random_configurations(fk, oracle, seed):
+    """Seeded random window sizes, defer blocks, grids, retained sets, GQA factors and ragged batches: every
+    step's attention output, the final planes and the counters against the oracle's WindowedUnit."""
+    from paper_2507_20030_b200 import synth
+    rng = np.random.default_rng(5000 + seed)
+    P = 1 << int(rng.integers(6, 12))
+    S, R = int(rng.integers(0, 9)), int(rng.integers(0, 13))
+    D = int(rng.choice([1, 1, 2, 3, 7, 16]))
+    GQ = int(rng.choice([1, 2, 4]))
+    H = int(rng.integers(1, 4))
+    HQ = H * GQ
+    B = int(rng.integers(1, 4))
+    M = int(rng.integers(1, min(P // 2 + 1, 40) + 1))
+    steps = int(rng.integers(3, 3 * max(D, 2) + 4))
+    Ts = [int(rng.integers(S + R + (1 if S + R == 0 else 0), S + R + P // 2 + 2)) for _ in range(B)]
+    dtype = torch.float32 if seed % 2 == 0 else torch.bfloat16
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
+                     prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R, n_defer=D)
+    mask = _random_mask(P, M, 31 * seed + 1)
+    mask[0] = 1
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    if S + R + (D if D > 1 else 0) == 0:
+        ctx.close()
+        pytest.skip("no window tensor in this draw")
+    wK, wV = ctx.alloc_window(B), ctx.alloc_window(B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    units = {}
+    for b, T in enumerate(Ts):
+        K, V = _make(900 + seed * 7 + b, 1, H, T, dtype)
+        V = (V * 0.25).to(dtype)
+        for h in range(H):
+            u = units[(b, h)] = oracle.WindowedUnit(P, bins, S, R, defer=D)
+            u.prefill(to_np64(K[0, h]), to_np64(V[0, h]))
+        ctx.prefill_windowed(0, K.cuda(), V.cuda(), cK[b:b + 1], cV[b:b + 1], wK[b:b + 1], wV[b:b + 1], t_len[b:b + 1])
+    out = torch.empty((B, HQ, 128), dtype=dtype, device="cuda")
+    for s_ in range(steps):
+        k, v = synth.make_token(91 + seed, s_, B, H, 128, pos=Ts[0] + s_, dtype=dtype)
+        v = (v * 0.25).to(dtype)
+        q = synth.make_q(91 + seed, s_, B, HQ, 128, dtype=dtype)
+        ctx.step_windowed(0, k.cuda(), v.cuda(), q.cuda(), cK, cV, wK, wV, t_len, out)
+        torch.cuda.synchronize()
+        got = to_np64(out)
+        for (b, h), u in units.items():
+            u.step(to_np64(k[b, h]), to_np64(v[b, h]))
+            want = u.attention(to_np64(q[b, h * GQ:(h + 1) * GQ]))
+            err = np.abs(got[b, h * GQ:(h + 1) * GQ] - want).max()
+            assert err <= ATTN_MAX_ABS, (seed, s_, b, h, err, (P, S, R, D, GQ, H, B, M, Ts))
+    assert t_len.tolist() == [T + steps for T in Ts] and ctx.device_status() == 0
+    gK, gV = to_np64(cK), to_np64(cV)
+    for (b, h), u in units.items():
+        assert np.abs(gK[b, h] - np.stack(u.CK)).max() <= 1e-4 * max(1.0, np.abs(np.stack(u.CK)).max())
+        assert np.abs(gV[b, h] - np.stack(u.CV)).max() <= 1e-4 * max(1.0, np.abs(np.stack(u.CV)).max())
+    ctx.close()
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("S,R,D", [(0, 0, 4), (3, 6, 5), (10, 50, 32)])
 def test_block_fold_is_bit_identical_to_single_token_updates(fk, dtype, S, R, D):
