@@ -64,7 +64,7 @@ typedef enum {
     FAEDKV_PREFILL_SIMT = 1,  /* float32 FMA contraction, twiddles exact to float32     */
     FAEDKV_PREFILL_UMMA = 2,  /* tcgen05 tensor-core contraction, bf16 operands, float32 accumulate */
     FAEDKV_PREFILL_FFT = 3    /* float32 two-pass FFT of every channel, then a gather of the retained
-                                 bins (power-of-two P; needs decode_mode AUTO or FFT): O(T log T) per
+                                 bins (power-of-two P; needs decode_mode AUTO, FFT or FFT_TWO_PASS): O(T log T) per
                                  channel instead of O(T * M), float32-exact                          */
 } faedkv_prefill_mode;
 
