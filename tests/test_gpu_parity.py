@@ -803,6 +803,50 @@ def test_block_fold_is_bit_identical_to_single_token_updates(fk, dtype, S, R, D)
         ctx.close()
 
 
+@pytest.mark.parametrize("defer", [1, 4])
+def test_windowed_step_replayed_as_a_cuda_graph(fk, defer):
+    """The windowed step uses up to three streams of the context (window attention beside the pass over C_K,
+    the second run of sequences of a call cut in two).  Captured into a CUDA graph and replayed, it must
+    give bit for bit what the same steps give when launched eagerly on a copy of the state."""
+    from paper_2507_20030_b200 import synth
+    P, M, B, H, HQ, S, R, T = 128, 24, 5, 8, 64, 3, 6, 40        # 320 columns: the call is cut into 2 + 3 sequences
+    dtype = torch.bfloat16
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B, kv_dtype=fk.BF16,
+                     prefill_mode=fk.PREFILL_SIMT, n_sink=S, n_recent=R, n_defer=defer)
+    ctx.plan(0, _random_mask(P, M, 9))
+    K, V = _make(321, B, H, T, dtype)
+    state = []
+    for _ in range(2):
+        cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+        wK, wV = ctx.alloc_window(B), ctx.alloc_window(B)
+        t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+        ctx.prefill_windowed(0, K.cuda(), V.cuda(), cK, cV, wK, wV, t_len)
+        state.append((cK, cV, wK, wV, t_len, torch.empty((B, HQ, 128), dtype=dtype, device="cuda")))
+    k, v = synth.make_token(7, 0, B, H, 128, pos=T, dtype=dtype)
+    q = synth.make_q(7, 0, B, HQ, 128, dtype=dtype)
+    k, v, q = k.cuda(), v.cuda(), q.cuda()
+    steps = 2 * defer + 3
+    cK, cV, wK, wV, t_len, out = state[0]
+    for _ in range(steps):                                        # eager
+        ctx.step_windowed(0, k, v, q, cK, cV, wK, wV, t_len, out)
+    torch.cuda.synchronize()
+    cK, cV, wK, wV, t_len, out = state[1]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            ctx.step_windowed(0, k, v, q, cK, cV, wK, wV, t_len, out, stream=side.cuda_stream)
+    torch.cuda.synchronize()
+    for _ in range(steps):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    for a, b in zip(state[0], state[1]):
+        assert torch.equal(a, b)
+    ctx.close()
+
+
 def test_windowed_rejects_short_prefill_and_non_fft_grids(fk):
     ctx = fk.Context(n_layers=1, n_kv_heads=1, n_q_heads=1, n_dft=100, max_batch=1, kv_dtype=fk.F32, n_sink=4, n_recent=8)
     ctx.plan(0, _mask_from_bins(100, [0, 1, 2]))
