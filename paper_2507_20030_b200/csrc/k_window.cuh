@@ -109,6 +109,7 @@ k_attn_window(const TQ *__restrict__ q, WindowArgs wa, const int32_t *__restrict
     const int t = t_len[b];
     const int first = win_folded(t + 1, S, wa.R, wa.D);       // offset (from S) of the oldest unfolded token
     const int W = S + (t + 1 - S - first);
+    const int slot0 = Rc > 0 ? first % Rc : 0;                // ring slot of the oldest unfolded token
     const TQ *kbase = winK + (size_t)bh * Wcap * kHeadDim + lane * 4, *vbase = winV + (size_t)bh * Wcap * kHeadDim + lane * 4;
     const TQ *kn = k_new + (size_t)bh * kHeadDim + lane * 4, *vn = v_new + (size_t)bh * kHeadDim + lane * 4;
     float m_run = -INFINITY, sum = 0.f;
@@ -121,7 +122,9 @@ k_attn_window(const TQ *__restrict__ q, WindowArgs wa, const int32_t *__restrict
             // row of the window tensor, or the step's new token
             const int n = first + w - S;             // offset from S of an unfolded token (w >= S)
             const bool is_new = w >= S && n == t - S;
-            const size_t off = (size_t)(w < S ? w : S + n % Rc) * kHeadDim;
+            int slot = slot0 + w - S;                // n mod Rc: at most Rc tokens wait, so one wrap at most
+            if (slot >= Rc) slot -= Rc;
+            const size_t off = (size_t)(w < S ? w : S + slot) * kHeadDim;
             kr[u] = Raw::load(is_new ? kn : kbase + off);
             vr[u] = Raw::load(is_new ? vn : vbase + off);
         }
