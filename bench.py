@@ -273,7 +273,7 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
         us = a.elapsed_time(b) / iters / NL * 1e3
         gbs = alg_bytes[name] / (us * 1e-6) / 1e9
         res[name] = {"us": us, "us_eager_launches": eager_us, "bytes": alg_bytes[name], "bound": "hbm", "achieved": gbs,
-                     "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"]}
+                     "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"], "frac_of_nominal_8000": gbs / 8000.0}
     if graphs:
         res["decode_us_per_layer_step"] = res["append_decode_attn"]["us"]
         res["decode_us_per_layer_step_two_calls"] = res["append"]["us"] + res["decode_attn"]["us"]
@@ -322,6 +322,7 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
         "us": us, "us_step_without_fold": sorted(per)[len(per) // 2], "us_step_with_fold": per[0], "defer": DEFER,
         "launch": "one CUDA graph per step of all layers" if graphs else "eager launches",
         "bytes": nbytes, "bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"],
+        "frac_of_nominal_8000": gbs / 8000.0,
         "what": "mean over 50 consecutive steps, the first of which folds 50 tokens into every layer's planes; "
                 "bytes = planes read once per step + read and written once per 50 steps"}
     if ctx2.device_status() != 0:
@@ -569,7 +570,7 @@ def run_ours(args):
         # float32 FMA pipe: 148 SMs x 128 lanes x 2 FLOP x 1.965 GHz
         peak_tf, bound = 148 * 128 * 2 * 1.965e9 / 1e12, "alu"
     roofline = {"kernel": "prefill transform (" + mode + ")", "bound": bound, "achieved": achieved_tf,
-                "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
+                "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf, "frac_of_nominal_2250": (achieved_tf / 2250.0) if bound == "tensor" else None,
                 # ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel at this size
                 # (profiles/k_prefill_umma_T32768_M4096.md); the kernel is unchanged since that capture
                 "traffic": 191.4e6 if (mode == "tcgen05-bf16" and (args.twiddle_terms or 1) == 1) else None,
