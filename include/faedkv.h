@@ -238,6 +238,17 @@ int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const vo
                          const void *q, int batch, float *coefK, float *coefV, void *winK,
                          void *winV, int32_t *t_len, float scale, void *out, void *stream);
 
+/* Eq. 13 written out: K_out, V_out [batch][n_kv_heads][L][head_dim] (kv_dtype) receive, per sequence, the
+ * cache the windowed attention attends over, in order: the S sink tokens, the reconstruction (Eq. 11) of
+ * the min(folded, P) positions of the transformed segment, the tokens still in the time domain (the last
+ * R; R .. R + D - 1 with the block-deferred fold), and zeros up to row L.  Rows past L are not written; a
+ * sequence longer than L is cut.  For callers that run their own attention on the reconstructed cache;
+ * faedkv_step_windowed itself never materialises these rows.  Call it between steps.  Needs the
+ * FFT-shaped path like the other windowed calls. */
+int faedkv_reconstruct_windowed(faedkv_ctx *ctx, int layer, const float *coefK, const float *coefV,
+                                const void *winK, const void *winV, const int32_t *t_len, int batch,
+                                int L, void *K_out, void *V_out, void *stream);
+
 /* ---- frequency ablation and bin selection (Sec. 3.2) -----------------------------------------------
  * The paper chooses each layer's retained bins once per model: the P two-sided bins are cut into C
  * contiguous chunks (C = 22 in the paper), each chunk is zeroed in turn in the DFT of the layer's K and

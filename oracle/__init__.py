@@ -281,12 +281,9 @@ class WindowedUnit:
                 append(self.CV[0], self.CV[1], self.P, self.bins, self.folded, v_old)
                 self.folded += 1
 
-    def attention(self, q: np.ndarray, scale: float | None = None) -> np.ndarray:
-        """Eq. 13 then Eq. 3: one softmax over [sink | reconstructed segment | unfolded recent tokens]."""
-        q = _f64arr(q)
-        d = q.shape[1]
-        if scale is None:
-            scale = 1.0 / np.sqrt(d)
+    def materialise(self) -> tuple[np.ndarray, np.ndarray]:
+        """Eq. 13: K^ = [K_sink ; K~ ; K_recent] and the same for V (Eq. 13's V row read with V~), the
+        reconstruction covering the min(folded, P) positions of the transformed segment."""
         L = min(self.folded, self.P)
         parts_k, parts_v = [self.sinkK], [self.sinkV]
         if L > 0:
@@ -297,6 +294,15 @@ class WindowedUnit:
             parts_v.append(np.stack(self.recentV))
         Kt = np.concatenate([p for p in parts_k if p.shape[0] > 0], axis=0)
         Vt = np.concatenate([p for p in parts_v if p.shape[0] > 0], axis=0)
+        return Kt, Vt
+
+    def attention(self, q: np.ndarray, scale: float | None = None) -> np.ndarray:
+        """Eq. 13 then Eq. 3: one softmax over [sink | reconstructed segment | unfolded recent tokens]."""
+        q = _f64arr(q)
+        d = q.shape[1]
+        if scale is None:
+            scale = 1.0 / np.sqrt(d)
+        Kt, Vt = self.materialise()
         return attention_dense(q, Kt, Vt, scale)
 
 

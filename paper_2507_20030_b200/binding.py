@@ -30,6 +30,7 @@ EXPORTS = [
     "faedkv_compress_prefill", "faedkv_append", "faedkv_reconstruct", "faedkv_decode_attn",
     "faedkv_append_decode_attn", "faedkv_chunk_range", "faedkv_ablation_bins", "faedkv_mask_from_scores", "faedkv_ablate",
     "faedkv_convert_state", "faedkv_window_bytes", "faedkv_prefill_windowed", "faedkv_step_windowed",
+    "faedkv_reconstruct_windowed",
     "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
 ]
 
@@ -107,6 +108,8 @@ def load() -> ctypes.CDLL:
     lib.faedkv_prefill_windowed.restype = _int
     lib.faedkv_step_windowed.argtypes = [_vp, _int, _vp, _vp, _vp, _int, _vp, _vp, _vp, _vp, _vp, ctypes.c_float, _vp, _vp]
     lib.faedkv_step_windowed.restype = _int
+    lib.faedkv_reconstruct_windowed.argtypes = [_vp, _int, _vp, _vp, _vp, _vp, _vp, _int, _int, _vp, _vp, _vp]
+    lib.faedkv_reconstruct_windowed.restype = _int
     lib.faedkv_device_status.argtypes = [_vp, _vp]
     lib.faedkv_device_status.restype = _int
     lib.faedkv_decode_attn_static.argtypes = [_int, _int, _int, _int, _vp, _int, _vp, _vp, _vp, _vp, _int,
@@ -337,6 +340,19 @@ class Context:
         self._check(self._lib.faedkv_step_windowed(
             self._h, layer, _ptr(k_new), _ptr(v_new), _ptr(q), batch, _ptr(coefK), _ptr(coefV), _ptr(winK),
             _ptr(winV), _ptr(t_len), float(scale), _ptr(out), _stream(stream)))
+
+    def reconstruct_windowed(self, layer, coefK, coefV, winK, winV, t_len, L: int, K_out=None, V_out=None, stream=None):
+        """[sink | reconstructed segment | tokens still in the time domain | zeros] as [batch, n_kv_heads, L, head_dim]."""
+        batch = t_len.shape[0]
+        shape = (batch, self.n_kv_heads, L, self.head_dim)
+        if K_out is None:
+            K_out = torch.empty(shape, dtype=self.torch_dtype, device=coefK.device)
+        if V_out is None:
+            V_out = torch.empty(shape, dtype=self.torch_dtype, device=coefK.device)
+        self._check(self._lib.faedkv_reconstruct_windowed(
+            self._h, layer, _ptr(coefK), _ptr(coefV), _ptr(winK), _ptr(winV), _ptr(t_len), batch, L, _ptr(K_out),
+            _ptr(V_out), _stream(stream)))
+        return K_out, V_out
 
     def launch_count(self) -> int:
         return int(self._lib.faedkv_launch_count(self._h))

@@ -483,7 +483,8 @@ int fft_opt_in(faedkv_ctx *ctx, K kernel, size_t bytes, unsigned int &done_mask,
 // FFT-shaped reconstruction of one tensor: pairs of (pass A, pass B) launches over runs of units.
 template <typename TOut>
 int launch_reconstruct_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const float *coef, const int32_t *t_len, int units,
-                                  int L, void *out, cudaStream_t st) {
+                                  int L, void *out, cudaStream_t st, ReconRows rows = ReconRows{0, -1, 0, 1}) {
+    if (rows.unit_rows < 0) rows.unit_rows = L;
     const faedkv_config &c = ctx->cfg;
     FftScratch &f = ctx->fs;
     constexpr int kOutKind = sizeof(TOut) == 2 ? 4 : 5;
@@ -511,7 +512,7 @@ int launch_reconstruct_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const flo
             const size_t smem = rfft_smem_b(g.lgN2, lgMT);
 #define CALL(LG)                                                                                         \
             rc = fft_opt_in(ctx, FFT_PICK_T(k_rfft_inv_b, LG, lgMT, TOut), smem, f.attr_mask[kOutKind], LG + ((lgMT) == fft::fast_lg_transforms(LG) ? 16 : 0));               \
-            if (rc == 0) FFT_PICK_T(k_rfft_inv_b, LG, lgMT, TOut)<<<grid, fft::kThreads, smem, st>>>(g, f.Yr, t_len, c.n_kv_heads, u0, L, static_cast<TOut *>(out), lgMT)
+            if (rc == 0) FFT_PICK_T(k_rfft_inv_b, LG, lgMT, TOut)<<<grid, fft::kThreads, smem, st>>>(g, f.Yr, t_len, c.n_kv_heads, u0, L, static_cast<TOut *>(out), lgMT, rows)
             FAEDKV_FFT_SWITCH(g.lgN2, 2, CALL)
 #undef CALL
             if (rc) return rc == FAEDKV_ERR_UNSUPPORTED ? fail(ctx, rc, "no FFT kernel for 2^%d rows", g.lgN2) : rc;
@@ -1263,6 +1264,53 @@ int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const vo
     if (c.kv_dtype == FAEDKV_BF16)
         return dispatch_attn_fft<__nv_bfloat16, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
     return dispatch_attn_fft<float, true>(ctx, *p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+}
+
+int faedkv_reconstruct_windowed(faedkv_ctx *ctx, int layer, const float *coefK, const float *coefV, const void *winK,
+                                const void *winV, const int32_t *t_len, int batch, int L, void *K_out, void *V_out,
+                                void *stream) {
+    const LayerPlan *p = nullptr;
+    if (int r = check_layer(ctx, layer, &p)) return r;
+    if (int r = check_batch(ctx, batch)) return r;
+    const faedkv_config &c = ctx->cfg;
+    const int S = c.n_sink, R = c.n_recent, D = c.n_defer, Rc = win_ring(R, D);
+    if (coefK == nullptr || coefV == nullptr || t_len == nullptr || K_out == nullptr || V_out == nullptr ||
+        (S + Rc > 0 && (winK == nullptr || winV == nullptr)))
+        return fail(ctx, FAEDKV_ERR_INVALID_ARG, "NULL tensor passed to faedkv_reconstruct_windowed");
+    if (L < 1) return fail(ctx, FAEDKV_ERR_SHAPE, "L = %d must be at least 1", L);
+    if (int r = check_ptrs(ctx, {coefK, coefV, winK, winV, K_out, V_out})) return r;
+    if (int r = check_tlen(ctx, t_len)) return r;
+    if (!ctx->use_fft)
+        return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "the windowed calls need the FFT-shaped path (P a power of two in [64, 2^19])");
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int units = batch * c.n_kv_heads;
+    // the reconstructed segment at rows [S, S + min(L - S, P)), zeros past its live positions ...
+    const int Lmid = L - S < c.n_dft ? L - S : c.n_dft;
+    if (Lmid > 0) {
+        const ReconRows rows{S, L, -(S + R), D > 1 ? D : 1};
+        for (int kv = 0; kv < 2; ++kv) {
+            const float *coef = kv == 0 ? coefK : coefV;
+            void *out = kv == 0 ? K_out : V_out;
+            int r = c.kv_dtype == FAEDKV_BF16
+                        ? launch_reconstruct_fft_tensor<__nv_bfloat16>(ctx, *p, coef, t_len, units, Lmid, out, st, rows)
+                        : launch_reconstruct_fft_tensor<float>(ctx, *p, coef, t_len, units, Lmid, out, st, rows);
+            if (r) return r;
+        }
+    }
+    // ... then the sink rows, the waiting tokens right behind the live positions, and zeros to the end
+    for (int kv = 0; kv < 2; ++kv) {
+        const void *win = kv == 0 ? winK : winV;
+        void *out = kv == 0 ? K_out : V_out;
+        const dim3 grid(L, units);
+        if (c.kv_dtype == FAEDKV_BF16)
+            k_window_place<__nv_bfloat16><<<grid, kHeadDim, 0, st>>>(static_cast<const __nv_bfloat16 *>(win), static_cast<__nv_bfloat16 *>(out),
+                                                                    t_len, c.n_kv_heads, L, S, R, D, Rc, c.n_dft);
+        else
+            k_window_place<float><<<grid, kHeadDim, 0, st>>>(static_cast<const float *>(win), static_cast<float *>(out), t_len,
+                                                            c.n_kv_heads, L, S, R, D, Rc, c.n_dft);
+        if (int r = launch_check(ctx, "k_window_place")) return r;
+    }
+    return FAEDKV_OK;
 }
 
 int faedkv_chunk_range(int n_dft, int n_chunks, int chunk, int *lo, int *hi) {

@@ -67,12 +67,20 @@ k_rfft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float *__r
     fft_rows<LG, (LGT >= 0 ? LGT + kLgCW : -1)>(lg_cols, xa, xb, tw, load, store);
 }
 
+// Where the reconstructed positions go: position n of a unit lands in row row0 + n of its unit_rows output rows;
+// live positions = min(q(t_len + t_add), P), q() rounding down to a multiple of t_quant (the transformed
+// segment of a windowed cache: t_add = -(S + R), t_quant = the defer block).
+struct ReconRows {
+    int row0, unit_rows, t_add, t_quant;
+};
+
 // grid = (N1 / MT, cols / 16); block = 256; dynamic smem = rfft_smem_b(lgN2, lgMT).
-// out: rows of the tensor, [units][Lrows][128]; H: kv heads per sequence (t_len index = unit / H).
+// out: rows of the tensor, [units][rows.unit_rows][128], Lrows positions written (zeros past the live ones);
+// H: kv heads per sequence (t_len index = unit / H).
 template <int LG, int LGT, typename TOut>
 __global__ void __launch_bounds__(fft::kThreads)
 k_rfft_inv_b(fft::Geometry g, const float2 *__restrict__ Y, const int32_t *__restrict__ t_len, int H, int unit0,
-             int Lrows, TOut *__restrict__ out, int lgMT_rt) {
+             int Lrows, TOut *__restrict__ out, int lgMT_rt, ReconRows rows) {
     const int lgMT = LGT >= 0 ? LGT : lgMT_rt;   // compile-time in the fast instances
     using namespace fft;
     constexpr int NF = 1 << LG;                      // = N2
@@ -86,9 +94,11 @@ k_rfft_inv_b(fft::Geometry g, const float2 *__restrict__ Y, const int32_t *__res
     __syncthreads();
     // the 16 columns of a CTA belong to one unit (128 channels per unit)
     const int unit = unit0 + (g0 >> 7);
-    const int t = t_len[unit / H];
+    int t = t_len[unit / H] + rows.t_add;
+    if (t < 0) t = 0;
+    if (rows.t_quant > 1) t = t / rows.t_quant * rows.t_quant;
     const int live = t < (int)g.P ? t : (int)g.P;
-    TOut *obase = out + (size_t)unit * Lrows * kHeadDim + (g0 & (kHeadDim - 1));
+    TOut *obase = out + ((size_t)unit * rows.unit_rows + rows.row0) * kHeadDim + (g0 & (kHeadDim - 1));
     auto load = [&](int k2, int cidx) {
         return Y[y_index(g, m1_0 + (cidx >> kLgCW), k2, g0 + (cidx & (kCW - 1)))];
     };

@@ -53,6 +53,32 @@ __global__ void k_window_fill(const T *__restrict__ K, const T *__restrict__ V, 
     winV[d_o] = V[so];
 }
 
+// Eq. 13 materialised: the rows of [sink | reconstructed segment | waiting tokens] that are NOT the reconstructed
+// segment (which the inverse transform writes at rows [S, S + live)).  Row n of a unit: n < S the sink token n;
+// S + live <= n < S + live + u the waiting tokens in order; zero from there to L.  t_len is at rest (no step
+// in flight): every token sits in its ring slot.
+// grid = (L, units); block = 128.
+template <typename T>
+__global__ void k_window_place(const T *__restrict__ win, T *__restrict__ out, const int32_t *__restrict__ t_len,
+                               int H, int L, int S, int R, int D, int Rc, int P) {
+    const int n = blockIdx.x, unit = blockIdx.y, c = threadIdx.x;
+    const int t = t_len[unit / H];
+    const int folded = win_folded(t, S, R, D);
+    const int live = folded < P ? folded : P;
+    const int u = t - S - folded;                    // waiting tokens
+    T *dst = out + ((size_t)unit * L + n) * kHeadDim + c;
+    const T *src = nullptr;
+    if (n < S) {
+        if (n < t) src = win + ((size_t)unit * (S + Rc) + n) * kHeadDim + c;
+    } else if (n < S + live) {
+        return;                                      // written by the inverse transform
+    } else if (n - S - live < u) {
+        src = win + ((size_t)unit * (S + Rc) + S + (folded + n - S - live) % Rc) * kHeadDim + c;   // u > 0 implies Rc > 0
+    }
+    if (src != nullptr) *dst = *src;
+    else store1(dst, 0.f);
+}
+
 // Attention over the time-domain tokens of one (sequence, kv head) for its GQ query heads, in the same
 // unnormalised form as a tile of the transformed segment: per column the maximum score m, the sum of
 // exp(s - m), and o_w[col][c] = sum_w exp(s_w - m) v_w[c].  Rows: the S sink tokens, then the unfolded tokens

@@ -561,6 +561,23 @@ def test_prefill_fft_matches_oracle(fk, oracle, dtype, P, T, M, B, H):
 
 
 # ----------------------------------------------------------------------------- sink + recent window
+def _check_materialised(fk, ctx, units, cK, cV, wK, wV, t_len, dtype):
+    """Eq. 13 written out by the library against the oracle: [sink | reconstruction | waiting tokens], zeros
+    behind; once with room to spare and once cut short."""
+    lens = {key: u.materialise()[0].shape[0] for key, u in units.items()}
+    for L in (max(lens.values()) + 3, max(1, min(lens.values()) - 2)):
+        Kh, Vh = ctx.reconstruct_windowed(0, cK, cV, wK, wV, t_len, L)
+        torch.cuda.synchronize()
+        gK, gV = to_np64(Kh), to_np64(Vh)
+        for (b, h), u in units.items():
+            for got, want in ((gK[b, h], u.materialise()[0]), (gV[b, h], u.materialise()[1])):
+                n = min(L, want.shape[0])
+                tol = 2e-4 * max(1.0, np.abs(want).max()) + (np.abs(want[:n]) * 2.0 ** -8 if dtype == torch.bfloat16 else 0.0)
+                assert np.all(np.abs(got[:n] - want[:n]) <= tol), (L, b, h, np.abs(got[:n] - want[:n]).max())
+                assert not got[n:].any()
+    assert ctx.device_status() == 0
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("P,T,M,B,H,HQ,S,R,steps", [
     (256, 200, 40, 2, 2, 8, 10, 50, 12),      # the paper's S = 10, R = 50; GQA 4
@@ -617,6 +634,7 @@ def test_windowed_step_matches_oracle(fk, oracle, dtype, P, T, M, B, H, HQ, S, R
             t = T + steps
             for j, n in enumerate(range(t - R, t)):
                 assert np.array_equal(gwK[b, h, S + (n - S) % R], u.recentK[j]), (b, h, n)
+    _check_materialised(fk, ctx, units, cK, cV, wK, wV, t_len, dtype)
     ctx.close()
 
 
@@ -687,6 +705,7 @@ def test_deferred_step_matches_oracle(fk, oracle, dtype, P, Ts, M, H, HQ, S, R, 
         for j, n in enumerate(range(first, t)):   # ring slot of token n is (n - S) mod (R + D)
             assert np.array_equal(gwK[b, h, S + (n - S) % Rc], u.recentK[j]), (b, h, n)
             assert np.array_equal(gwV[b, h, S + (n - S) % Rc], u.recentV[j]), (b, h, n)
+    _check_materialised(fk, ctx, units, cK, cV, wK, wV, t_len, dtype)
     ctx.close()
 
 

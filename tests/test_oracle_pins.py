@@ -523,6 +523,8 @@ def test_deferred_all_bins_is_full_attention(oracle, S, R, D):
         got = u.attention(q, 0.3)
         want = _numpy_attention(q, K[:T + s], V[:T + s], 0.3)
         assert np.abs(got - want).max() < 1e-11, (s, np.abs(got - want).max())
+        Kh, Vh = u.materialise()                 # Eq. 13 written out: here, the cache itself
+        assert np.abs(Kh - K[:T + s]).max() < 1e-11 and np.abs(Vh - V[:T + s]).max() < 1e-11
         assert u.folded % D == 0 and R <= len(u.recentK) < R + D and u.folded + len(u.recentK) + S == u.t
         if s < steps:
             before = u.folded
