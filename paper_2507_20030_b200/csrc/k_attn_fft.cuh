@@ -13,6 +13,8 @@
 //
 // The scores never leave shared memory; the only intermediates in (L2-resident) global memory are the
 // two-pass arrays Y, Zf of P/2 complex values per column and the per-tile softmax statistics.
+// For P <= 16384 the three kernels of (2)-(4) are replaced by one kernel per column (k_attn_col.cuh), which
+// hands (5) ready weights Wg instead of Zf; (1) then writes Qs column-major.
 #pragma once
 #include "common.cuh"
 #include "k_attn.cuh"
