@@ -138,7 +138,7 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------------------- reference arm
 def _oracle_units_seconds(orc, torch, synth, n_units, T, P, bins, seed):
-    """Time the oracle's pruned DFT of `n_units` units (kv heads of layer 0, K) over all retained bins."""
+    """Time the oracle's pruned DFT of `n_units` units (kv heads of layer 0, K) over the bins given."""
     K, _ = synth.make_kv(seed, 1, n_units, T, 128, dtype=torch.bfloat16)
     x = K[0].double().numpy()
     t0 = time.perf_counter()
@@ -146,9 +146,75 @@ def _oracle_units_seconds(orc, torch, synth, n_units, T, P, bins, seed):
     return time.perf_counter() - t0
 
 
-def cpu_baseline(target_s: float = 12.0) -> dict:
-    """Oracle prefill throughput on the host cores, from a bounded sample extrapolated over the
-    independent (layer, head, tensor) units of the workload."""
+def _cpu_config0(orc, torch, synth):
+    """configs[0] in full on the oracle: prefill of the 16 units, 64 appends, reconstruction (seconds each)."""
+    import numpy as np
+    P = T = 2048
+    M, H, steps = 256, 8, 64
+    seed = synth.config_seed(0, 0)
+    bins = orc.plan(P, orc.mask_lowpass(P, M))
+    K, V = synth.make_kv(seed, 1, H, T, 128, dtype=torch.float32)
+    xs = [K[0].double().numpy(), V[0].double().numpy()]
+    t0 = time.perf_counter()
+    planes = [orc.compress(x, P, bins) for x in xs]
+    t1 = time.perf_counter()
+    toks = [synth.make_token(seed, s_, 1, H, 128, pos=T + s_, dtype=torch.float32) for s_ in range(steps)]
+    toks = [(k[0].double().numpy(), v[0].double().numpy()) for k, v in toks]
+    planes = [(np.ascontiguousarray(re), np.ascontiguousarray(im)) for re, im in planes]
+    t2 = time.perf_counter()
+    for s_ in range(steps):
+        for kv in range(2):
+            for h in range(H):
+                orc.append(planes[kv][0][h], planes[kv][1][h], P, bins, T + s_, toks[s_][kv][h])
+    t3 = time.perf_counter()
+    for kv in range(2):
+        for h in range(H):
+            orc.reconstruct(planes[kv][0][h], planes[kv][1][h], P, bins, P)
+    t4 = time.perf_counter()
+    return {"what": "configs[0] in full: prefill of 2 x 8 units (2048 tokens, 256 bins), 64 appends, reconstruct L = 2048",
+            "prefill_s": t1 - t0, "appends_s": t3 - t2, "reconstruct_s": t4 - t3, "total_s": (t1 - t0) + (t3 - t2) + (t4 - t3),
+            "prefill_tokens_per_s": T / (t1 - t0), "append_us_per_step": (t3 - t2) / steps * 1e6}
+
+
+def _cpu_decode_slice(orc, torch, synth, DW, rows_cap=2048):
+    """One unit slice of the decode calls at a decode workload's shape: 8 appends of one (sequence, kv head)'s K
+    planes, the reconstruction of `rows_cap` of its rows and decode attention of the kv head's query heads over
+    `rows_cap` positions; each scaled linearly to a layer-step of the workload (units and rows are independent)."""
+    import numpy as np
+    P = T = DW["T"]
+    M, H, HQ, B = DW["M"], DW["n_kv_heads"], DW["n_q_heads"], DW["batch"]
+    seed = synth.config_seed(DW["config"])
+    bins = orc.plan(P, orc.mask_mixed(P, M, 0, seed))
+    rng = np.random.default_rng(seed)
+    re, im = rng.standard_normal((M, 128)) * np.sqrt(T), rng.standard_normal((M, 128)) * np.sqrt(T)
+    vre, vim = rng.standard_normal((M, 128)) * np.sqrt(T), rng.standard_normal((M, 128)) * np.sqrt(T)
+    x = rng.standard_normal(128)
+    t0 = time.perf_counter()
+    for s_ in range(8):
+        orc.append(re, im, P, bins, T + s_, x)
+    t_app = (time.perf_counter() - t0) / 8
+    rows = min(rows_cap, P)
+    t0 = time.perf_counter()
+    orc.reconstruct(re, im, P, bins, rows)
+    t_rec = time.perf_counter() - t0
+    G = HQ // H
+    q = rng.standard_normal((G, 128))
+    t0 = time.perf_counter()
+    orc.decode_attn(q, re / T, im / T, vre, vim, P, bins, rows)
+    t_att = time.perf_counter() - t0
+    units = B * H
+    return {"workload": DW["name"], "extrapolated": True,
+            "slice": f"1 of {units} (sequence, kv head) units; {rows} of {P} positions for reconstruct / attention",
+            "slice_seconds": {"append_one_tensor": t_app, "reconstruct_one_tensor": t_rec, "decode_attn": t_att},
+            "append_us_per_layer_step": t_app * 2 * units * 1e6,
+            "reconstruct_ms_per_layer": t_rec * (P / rows) * 2 * units * 1e3,
+            "decode_attn_us_per_layer_step": t_att * (P / rows) * units * 1e6}
+
+
+def cpu_baseline(target_s: float = 10.0, extras: bool = True) -> dict:
+    """Oracle prefill throughput on the host cores, from a bounded sample extrapolated over the independent
+    (layer, head, tensor) units of the workload; with `extras` also the same on one thread, configs[0] in full and
+    a unit slice of the decode calls at the streaming-decode shape."""
     import torch
     import oracle as orc
     from paper_2507_20030_b200 import synth
@@ -156,6 +222,7 @@ def cpu_baseline(target_s: float = 12.0) -> dict:
     W = WORKLOAD
     P = T = W["T"]
     cores = len(os.sched_getaffinity(0))
+    orc.set_threads(cores)
     bins = orc.plan(P, orc.mask_mixed(P, W["M"], 0, synth.config_seed(W["config"])))
     seed = synth.config_seed(W["config"], 0)
     t1 = _oracle_units_seconds(orc, torch, synth, 1, T, P, bins, seed)
@@ -163,10 +230,23 @@ def cpu_baseline(target_s: float = 12.0) -> dict:
     t_sample = t1 if n_units == 1 else _oracle_units_seconds(orc, torch, synth, n_units, T, P, bins, seed)
     units = W["n_layers"] * W["batch"] * W["n_kv_heads"] * 2            # (layer, head, K|V)
     full_s = t_sample * units / n_units
-    return {"value": W["batch"] * T / full_s, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": (f"pruned DFT of {n_units} of {units} units (layer 0, kv heads 0..{n_units - 1}, K): all {T} tokens "
-                       f"x 128 channels x {W['M']} bins in {t_sample:.2f} s; extrapolated linearly over units"),
-            "sample_seconds": t_sample}
+    res = {"value": W["batch"] * T / full_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": (f"pruned DFT of {n_units} of {units} units (layer 0, kv heads 0..{n_units - 1}, K): all {T} tokens "
+                      f"x 128 channels x {W['M']} bins in {t_sample:.2f} s; extrapolated linearly over units"),
+           "sample_seconds": t_sample}
+    if extras:
+        # one thread: every 8th retained bin of one unit (bins are independent loops of equal cost)
+        orc.set_threads(1)
+        sub = bins[::8]
+        t_one = _oracle_units_seconds(orc, torch, synth, 1, T, P, sub, seed)
+        full_one = t_one * (len(bins) / len(sub)) * units
+        res["one_thread"] = {"value": W["batch"] * T / full_one, "unit": UNIT, "cores": 1,
+                             "sample": f"{len(sub)} of {len(bins)} bins of 1 unit in {t_one:.2f} s; extrapolated linearly over bins and units",
+                             "sample_seconds": t_one}
+        orc.set_threads(cores)
+        res["config0_full"] = _cpu_config0(orc, torch, synth)
+        res["decode_slices"] = [_cpu_decode_slice(orc, torch, synth, DECODE_WORKLOADS[0])]
+    return res
 
 
 def run_reference(args):
@@ -177,7 +257,7 @@ def run_reference(args):
     vals = []
     base = None
     for i in range(args.warmup + args.steps):
-        base = cpu_baseline(target_s=max(2.0, min(12.0, 90.0 / max(1, args.warmup + args.steps))))
+        base = cpu_baseline(target_s=max(2.0, min(12.0, 90.0 / max(1, args.warmup + args.steps))), extras=False)
         if i >= args.warmup:
             vals.append(base)
     v = statistics.mean(b["value"] for b in vals)
@@ -193,6 +273,31 @@ def run_reference(args):
 
 
 
+# --------------------------------------------------------------------------------------- profiler figures
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the prefill contraction at the bench
+# size, from a profiler capture, together with the hash of the kernel source the capture was taken from.  The
+# figure is reported only while the kernel source still hashes to that value; after any change to the kernel it
+# reads null until the capture is repeated.
+PREFILL_TRAFFIC = {"bytes": 191.4e6, "kernel_sha256_16": "4db284614b54b599", "captured": "2026-11-27"}
+
+
+def _kernel_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("k_prefill_umma.cuh", "umma_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2507_20030_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def prefill_kernel_traffic():
+    cur = _kernel_hash()
+    if PREFILL_TRAFFIC["bytes"] is not None and PREFILL_TRAFFIC["kernel_sha256_16"] == cur:
+        return PREFILL_TRAFFIC["bytes"], (f"ncu capture of {PREFILL_TRAFFIC['captured']}, one launch at this size; "
+                                          f"kernel source sha256 {cur}")
+    return None, f"kernel source (sha256 {cur}) has changed since the last profiler capture"
+
+
 # --------------------------------------------------------------------------------------- decode sections
 DECODE_WORKLOADS = [
     dict(name="configs[2]: streaming decode, batch 16, prefill 16384 tokens at 1/8 retention", config=2,
@@ -202,6 +307,18 @@ DECODE_WORKLOADS = [
     dict(name="configs[4] cell: 32 kv = 32 query heads, batch 32, 4096 tokens at 1/8 retention", config=4,
          n_layers=32, n_kv_heads=32, n_q_heads=32, batch=32, T=4096, M=512),
 ]
+
+
+def recon_alu_roofline(P, n_cols, seconds):
+    """The reconstruction as float32 arithmetic: a real inverse FFT of length P per channel is a complex FFT of
+    N = P/2 points, 5 N log2 N flop, against the float32 FMA peak 148 SMs x 128 lanes x 2 x 1.965 GHz.  At the
+    bench sizes this floor is level with the HBM floor, so both fractions are reported."""
+    N = P // 2
+    flop = 5.0 * N * (N.bit_length() - 1) * n_cols
+    peak = 148 * 128 * 2 * 1.965e9 / 1e12
+    tf = flop / seconds / 1e12
+    return {"bound": "alu", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+            "flop_model": "5 N log2 N per channel, N = P/2"}
 
 
 def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
@@ -216,13 +333,29 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     cKs, cVs, tls = [], [], []
     for l in range(NL):
         ctx.plan(l, binding.mask_mixed(P, M, l, seed))
+    prefill_ms = []
+    for l in range(NL):
         K, V = synth.make_kv(synth.config_seed(W["config"], l), B, H, T, D, dtype=torch.bfloat16, device=dev)
         cK, cV = ctx.alloc_coef(l, B, device=dev), ctx.alloc_coef(l, B, device=dev)
         tl = torch.zeros(B, dtype=torch.int32, device=dev)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
         ctx.compress_prefill(l, K, V, cK, cV, tl)
+        b.record()
         cKs.append(cK); cVs.append(cV); tls.append(tl)
         torch.cuda.synchronize()
+        prefill_ms.append(a.elapsed_time(b))
         del K, V
+    # the state's own prefill (tensor-core contraction), one launch per layer; the first layers warm the kernel up
+    pf = sorted(prefill_ms[min(2, NL - 1):])
+    pf_ms = pf[len(pf) // 2]
+    pf_flop = 2.0 * (2 * M) * T * (B * H * D) * 2
+    prefill = {"ms_per_layer": pf_ms, "tokens_per_s": B * T / (pf_ms * 1e-3 * NL), "flop_per_layer": pf_flop,
+               "bound": "tensor", "achieved": pf_flop / (pf_ms * 1e-3) / 1e12, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+               "frac": pf_flop / (pf_ms * 1e-3) / 1e12 / peaks["bf16_sustained"],
+               "frac_of_burst": pf_flop / (pf_ms * 1e-3) / 1e12 / peaks["bf16"],
+               "what": "median over layers of the event-timed faedkv_compress_prefill that builds this section's state"}
     k_new, v_new = synth.make_token(seed, 0, B, H, D, pos=T, dtype=torch.bfloat16, device=dev)
     q = synth.make_q(seed, 0, B, HQ, D, dtype=torch.bfloat16, device=dev)
     out = torch.empty((B, HQ, D), dtype=torch.bfloat16, device=dev)
@@ -238,7 +371,12 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     coef_bytes = 2 * B * H * 2 * M * D * 4                      # K and V planes of one layer
     alg_bytes = {"append": 2 * coef_bytes, "decode_attn": coef_bytes, "append_decode_attn": 2 * coef_bytes,
                  "step_windowed": 2 * coef_bytes}
-    res = {"workload": W["name"], "iters": iters, "planes_bytes_per_layer": coef_bytes,
+    if not W.get("no_reconstruct"):
+        Ko = torch.empty((B, H, P, D), dtype=torch.bfloat16, device=dev)
+        Vo = torch.empty_like(Ko)
+        loops["reconstruct"] = lambda: [ctx.reconstruct(l, cKs[l], cVs[l], tls[l], P, Ko, Vo) for l in range(NL)]
+        alg_bytes["reconstruct"] = coef_bytes + 2 * B * H * P * D * 2          # planes in + bf16 rows out
+    res = {"workload": W["name"], "iters": iters, "planes_bytes_per_layer": coef_bytes, "prefill": prefill,
            "l2": "32 layers cycled: %.0f MiB of planes per layer" % (coef_bytes / 2 ** 20)}
     side = torch.cuda.Stream()
     for name, fn in loops.items():
@@ -274,6 +412,8 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
         gbs = alg_bytes[name] / (us * 1e-6) / 1e9
         res[name] = {"us": us, "us_eager_launches": eager_us, "bytes": alg_bytes[name], "bound": "hbm", "achieved": gbs,
                      "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"], "frac_of_nominal_8000": gbs / 8000.0}
+        if name == "reconstruct":
+            res[name]["alu"] = recon_alu_roofline(P, 2 * B * H * D, us * 1e-6)
     if graphs:
         res["decode_us_per_layer_step"] = res["append_decode_attn"]["us"]
         res["decode_us_per_layer_step_two_calls"] = res["append"]["us"] + res["decode_attn"]["us"]
@@ -334,6 +474,100 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     del cKs, cVs
     torch.cuda.empty_cache()
     return res
+
+
+# --------------------------------------------------------------------------------------- configs[4] sweep
+def sweep_cells():
+    """The 48 cells of the retention / batch sweep on the MHA cache (32 kv = 32 query heads)."""
+    cells = []
+    for T in (4096, 16384):
+        for B in (1, 8, 32):
+            for r_den in (4, 8, 16, 32):
+                for mask in ("lowpass", "mixed"):
+                    cells.append(dict(T=T, batch=B, r_den=r_den, M=T // r_den, mask=mask))
+    return cells
+
+
+def sweep_section(torch, binding, synth, dev, peaks, cells, iters=5):
+    """Per cell: the prefill through both routes (tensor-core contraction, FFT-shaped) and the fused decode step
+    (CUDA graph over the cell's layers).  A cell uses as many layers as make its planes exceed twice the L2
+    (at least 4, at most 32), so that no layer's planes survive in L2 between steps."""
+    H = HQ = 32
+    D = 128
+    out_cells = []
+    seed = synth.config_seed(4)
+    side = torch.cuda.Stream()
+    for c in cells:
+        T, B, M = c["T"], c["batch"], c["M"]
+        P = T
+        coef_bytes = 2 * B * H * 2 * M * D * 4                  # K and V planes of one layer
+        NL = int(min(32, max(4, -(-2 * 126 * 2 ** 20 // coef_bytes))))
+        ctxs = {}
+        for route, mode in (("gemm", binding.PREFILL_UMMA), ("fft", binding.PREFILL_FFT)):
+            ctxs[route] = binding.Context(n_layers=NL, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=B,
+                                          kv_dtype=binding.BF16, prefill_mode=mode)
+            for l in range(NL):
+                m = binding.mask_lowpass(P, M) if c["mask"] == "lowpass" else binding.mask_mixed(P, M, l, seed)
+                ctxs[route].plan(l, m)
+        kv_bytes = 2 * B * H * T * D * 2
+        n_kv = NL if kv_bytes * NL <= (2 << 30) else 1          # small caches: one per layer, so that none is L2-resident
+        KV = [synth.make_kv(seed + 31 * l + T + B, B, H, T, D, dtype=torch.bfloat16, device=dev) for l in range(n_kv)]
+        cKs = [ctxs["gemm"].alloc_coef(l, B, device=dev) for l in range(NL)]
+        cVs = [ctxs["gemm"].alloc_coef(l, B, device=dev) for l in range(NL)]
+        tls = [torch.zeros(B, dtype=torch.int32, device=dev) for _ in range(NL)]
+        ms = {}
+        for route in ("fft", "gemm"):                             # the contraction last: its planes are the decode state
+            ctx = ctxs[route]
+            run = lambda: [ctx.compress_prefill(l, KV[l % n_kv][0], KV[l % n_kv][1], cKs[l], cVs[l], tls[l]) for l in range(NL)]
+            run()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            run()
+            b.record()
+            torch.cuda.synchronize()
+            ms[route] = a.elapsed_time(b) / NL
+        ctx = ctxs["gemm"]
+        k_new, v_new = synth.make_token(seed, 0, B, H, D, pos=T, dtype=torch.bfloat16, device=dev)
+        q = synth.make_q(seed, 0, B, HQ, D, dtype=torch.bfloat16, device=dev)
+        out = torch.empty((B, HQ, D), dtype=torch.bfloat16, device=dev)
+        fn = lambda: [ctx.append_decode_attn(l, k_new, v_new, q, cKs[l], cVs[l], tls[l], out) for l in range(NL)]
+        graph = torch.cuda.CUDAGraph()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+            side.synchronize()
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.synchronize()
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(iters):
+            graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) / iters / NL * 1e3
+        gbs = 2 * coef_bytes / (us * 1e-6) / 1e9
+        flop = 2.0 * (2 * M) * T * (B * H * D) * 2
+        for cx in ctxs.values():
+            if cx.device_status() != 0:
+                raise RuntimeError("a kernel reported a device-side timeout; the numbers are invalid")
+            cx.close()
+        out_cells.append({"T": T, "B": B, "r": f"1/{c['r_den']}", "M": M, "mask": c["mask"], "layers": NL,
+                          "fused_us": round(us, 2), "fused_frac": round(gbs / peaks["hbm"], 4),
+                          "gemm_ms": round(ms["gemm"], 4), "gemm_tflops": round(flop / (ms["gemm"] * 1e-3) / 1e12, 1),
+                          "fft_ms": round(ms["fft"], 4), "fft_tok_s": round(B * T / (ms["fft"] * 1e-3)),
+                          "gemm_tok_s": round(B * T / (ms["gemm"] * 1e-3)),
+                          "faster_prefill": "gemm" if ms["gemm"] < ms["fft"] else "fft"})
+        del KV, cKs, cVs
+        torch.cuda.empty_cache()
+    return {"what": "configs[4]: MHA cache (32 kv = 32 query heads, 32-layer model; per cell the layers that are cycled are listed), "
+                    "fused step = faedkv_append_decode_attn us per layer (CUDA graph), frac = planes read + written / measured HBM peak; "
+                    "prefill ms per layer through the tensor-core contraction and through the FFT-shaped route",
+            "cells": out_cells}
 
 # --------------------------------------------------------------------------------------- our arm
 def run_ours(args):
@@ -551,6 +785,12 @@ def run_ours(args):
         torch.cuda.empty_cache()
         for DW in DECODE_WORKLOADS:
             decode_sections.append(decode_section(torch, binding, synth, dev, DW, peaks, args.decode_config_iters))
+    sweep = None
+    if not args.no_sweep and not args.no_decode_configs and not args.layers:
+        cells = sweep_cells()
+        if args.sweep_cells:
+            cells = cells[:args.sweep_cells]
+        sweep = sweep_section(torch, binding, synth, dev, peaks, cells)
     barrier()
 
     if rank != 0:
@@ -564,6 +804,9 @@ def run_ours(args):
     prefill_launch_ms = total_ms("prefill") / len(rec["prefill"])
     achieved_tf = flop_per_launch / (prefill_launch_ms * 1e-3) / 1e12
     mode = "simt-f32" if args.prefill_mode == binding.PREFILL_SIMT else "tcgen05-bf16"
+    traffic, traffic_source = None, "no profiler capture for this mode"
+    if mode == "tcgen05-bf16" and (args.twiddle_terms or 1) == 1:
+        traffic, traffic_source = prefill_kernel_traffic()
     if mode == "tcgen05-bf16":
         peak_tf, bound = peaks["bf16_sustained"], "tensor"
     else:
@@ -571,9 +814,7 @@ def run_ours(args):
         peak_tf, bound = 148 * 128 * 2 * 1.965e9 / 1e12, "alu"
     roofline = {"kernel": "prefill transform (" + mode + ")", "bound": bound, "achieved": achieved_tf,
                 "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf, "frac_of_nominal_2250": (achieved_tf / 2250.0) if bound == "tensor" else None,
-                # ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel at this size
-                # (profiles/k_prefill_umma_T32768_M4096.md); the kernel is unchanged since that capture
-                "traffic": 191.4e6 if (mode == "tcgen05-bf16" and (args.twiddle_terms or 1) == 1) else None,
+                "traffic": traffic, "traffic_source": traffic_source,
                 "peak_source": peaks["source"] + (" bf16 sustained" if bound == "tensor" else " (derived f32 FMA peak)"),
                 "flop_per_launch": flop_per_launch, "launch_ms": prefill_launch_ms,
                 "mma_passes": (args.twiddle_terms if args.twiddle_terms else 1) if bound == "tensor" else None}
@@ -599,7 +840,8 @@ def run_ours(args):
         "reconstruct": {"us": recon_ms * 1e3, "bytes": coef_bytes + 2 * B * H * P * D * 2, "bound": "hbm",
                         "achieved": (coef_bytes + 2 * B * H * P * D * 2) / (recon_ms * 1e-3) / 1e9, "peak": peaks["hbm"],
                         "unit": "GB/s", "frac": (coef_bytes + 2 * B * H * P * D * 2) / (recon_ms * 1e-3) / 1e9 / peaks["hbm"],
-                        "what": "FFT-shaped (float32 two-pass FFT per channel); instruction-bound, bytes = planes in + bf16 rows out",
+                        "alu": recon_alu_roofline(P, 2 * B * H * D, recon_ms * 1e-3),
+                        "what": "FFT-shaped (float32 FFT per channel); bytes = planes in + bf16 rows out",
                         "dense_equivalent_tflops": 2.0 * P * (2 * M) * n_c * 2 / (recon_ms * 1e-3) / 1e12},
         "decode_iters": n_dec,
     }
@@ -620,8 +862,25 @@ def run_ours(args):
                        "multi_gpu": "replicas only"},
             "phase_ms": phase_ms, "prefill_ms": prefill_ms,
             "roofline": roofline, "prefill_fft": prefill_fft, "decode": decode, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
+    line["sweep"] = sweep
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
+    # compact last key, so that a truncated record of the line still carries every headline figure:
+    # [us per layer-step, fraction of the measured HBM peak] per call and workload; prefill [TFLOP/s, fraction of
+    # the measured sustained bf16 peak]
+    def pair(d):
+        return [round(d["us"], 1), round(d["frac"], 3)]
+    summary = {"unit": "[us/layer/step, frac of measured HBM peak]; prefill: [TFLOP/s, frac of measured sustained bf16 peak]",
+               "cfg1": {"prefill": [round(achieved_tf, 1), round(achieved_tf / peak_tf, 3)], "append": pair(decode["append"]),
+                        "attn": pair(decode["decode_attn"]), "fused": pair(decode["append_decode_attn"]),
+                        "recon": pair(decode["reconstruct"])}}
+    for key, sec in zip(("cfg2", "cfg3", "cfg4cell"), decode_sections):
+        summary[key] = {"prefill": [round(sec["prefill"]["achieved"], 1), round(sec["prefill"]["frac"], 3)],
+                        "append": pair(sec["append"]), "attn": pair(sec["decode_attn"]), "fused": pair(sec["append_decode_attn"]),
+                        "win": pair(sec["step_windowed"]), "defer": pair(sec["step_windowed_deferred"])}
+        if "reconstruct" in sec:
+            summary[key]["recon"] = pair(sec["reconstruct"])
+    line["decode_summary"] = summary
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -648,6 +907,8 @@ def main():
                     help="profiling case: run only the decode section of configs[2] or configs[3] (eager launches; "
                          "combine with --layers and --decode-config-iters 1)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the configs[4] retention / batch sweep")
+    ap.add_argument("--sweep-cells", type=int, default=0, help="run only the first N cells of the sweep")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

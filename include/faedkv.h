@@ -4,9 +4,11 @@
  * The library keeps an LLM KV cache compressed as the retained bins of its
  * discrete Fourier transform along the token axis (FAEDKV, Sec. 4).  It owns
  * three things and nothing else: the per-layer bin plan, small device tables
- * derived from it, and a fixed scratch area sized at faedkv_create().  Every
- * tensor, every coefficient plane and every token counter belongs to the
- * caller.
+ * derived from it, and a scratch area that is sized while layers are planned
+ * (faedkv_plan() allocates it on the first plan and re-allocates the parts
+ * that depend on the bin count whenever a plan brings a larger M than any
+ * before it; no other call allocates).  Every tensor, every coefficient plane
+ * and every token counter belongs to the caller.
  *
  * Conventions
  *   P        DFT grid size (the paper's N / N_DFT), fixed at create time.
@@ -26,8 +28,9 @@
  * Pointers are DEVICE pointers unless a comment says "host".  Tensor and
  * coefficient pointers must be 16-byte aligned, t_len 4-byte aligned.  Calls
  * validate their arguments on the
- * host and enqueue work on `stream`; they do not synchronise and do not
- * allocate.  Return value: 0 on success, a negative faedkv_status otherwise;
+ * host and enqueue work on `stream`; apart from faedkv_create(), faedkv_plan()
+ * and faedkv_device_status() they do not synchronise and do not allocate.
+ * Return value: 0 on success, a negative faedkv_status otherwise;
  * faedkv_last_error() gives the text of the last failure on that context.
  * There is no CPU fallback: what the kernels do not support is an error.
  * A context must not be used from two host threads at once.
@@ -84,7 +87,8 @@ typedef enum {
 typedef struct {
     int n_layers;      /* >= 1                                                     */
     int n_kv_heads;    /* >= 1                                                     */
-    int n_q_heads;     /* multiple of n_kv_heads, at most 8 query heads per kv head */
+    int n_q_heads;     /* multiple of n_kv_heads; 1 to 8 query heads per kv head (any value:
+                          e.g. 7 for a 28 / 4 grouped-query model)                  */
     int head_dim;      /* must be 128                                              */
     int n_dft;         /* P >= 2; need not be a power of two                       */
     int max_batch;     /* >= 1; sizes the scratch area                             */
@@ -102,8 +106,10 @@ typedef struct {
                           2 .. 128 = block-deferred fold, see the window section       */
 } faedkv_config;
 
-/* Create a context on the CURRENT CUDA device.  Allocates the scratch area
- * (a few floats per (batch, query head, position of the grid)).  host: cfg, out. */
+/* Create a context on the CURRENT CUDA device.  Allocates only a few counters; the scratch area
+ * (a few floats per (batch, query head, position of the grid) and per retained bin) is allocated
+ * by faedkv_plan().  max_batch * n_kv_heads and max_batch * n_q_heads / 16 must not exceed 65535 (they
+ * index a grid dimension).  host: cfg, out. */
 int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out);
 
 /* Free the context, its plans and its scratch.  NULL is allowed. */
@@ -117,7 +123,12 @@ const char *faedkv_last_error(const faedkv_ctx *ctx);
  * length P/2 + 1): nonzero = retain one-sided bin k and, implicitly, its
  * mirror P-k.  Builds the ascending bin list and its device copy; replaces an
  * earlier plan of the same layer (the caller must not have work of that layer
- * in flight).  *n_bins_out (host, may be NULL) receives M.  M = 0 is an error. */
+ * in flight).  *n_bins_out (host, may be NULL) receives M.  M = 0 is an error.
+ * Allocates, and synchronises the device: the first plan of a context sizes the
+ * scratch area, and a plan whose M exceeds every earlier M of the context frees
+ * and re-allocates the M-dependent parts of it -- buffers that calls of OTHER
+ * layers in flight may still be using.  So plan all layers before the first
+ * transform call, or make sure the context has no work in flight when planning. */
 int faedkv_plan(faedkv_ctx *ctx, int layer, const uint8_t *bin_mask, int *n_bins_out);
 
 /* Number of retained bins of a planned layer, or a negative status. */
@@ -173,8 +184,10 @@ int faedkv_reconstruct(faedkv_ctx *ctx, int layer, const float *coefK, const flo
 /* Decode attention (Eq. 3 on the reconstruction of Eq. 11):
  *   out[g] = softmax_n( scale * q[g] . K~[n] ) * V~,  n < min(t_len[b], P)
  * evaluated in the frequency domain, without writing K~ or V~ to memory.
- * scale = 0 means 1/sqrt(head_dim).  Uses the context's scratch area: two
- * calls on the same context must not overlap on the GPU. */
+ * scale = 0 means 1/sqrt(head_dim).  A sequence with t_len[b] = 0 has no token
+ * to attend to: its rows of out are written as zero (the empty sum of Eq. 3).
+ * Uses the context's scratch area: two calls on the same context must not
+ * overlap on the GPU. */
 int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *coefK,
                        const float *coefV, const int32_t *t_len, int batch, float scale,
                        void *out, void *stream);
@@ -233,7 +246,11 @@ int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const voi
  * reconstruction of min(folded(t + 1), P) positions and all waiting tokens including the new one,
  * then the new token takes its ring slot and t_len[b] += 1.
  * Needs the FFT-shaped decode path (P a power of two in [64, 2^19]); FAEDKV_ERR_UNSUPPORTED
- * otherwise.  winK, winV, coefK, coefV and t_len are updated in place. */
+ * otherwise.  The segment Eq. 10 transforms, N - S - R tokens, is rarely a power of two: create the
+ * context with n_dft = the next power of two at or above the longest segment that must not alias
+ * (e.g. 16324 tokens of a 16384-token prompt on P = 16384); positions the segment has not reached yet
+ * are masked out of the softmax, so a grid longer than the segment changes no result.
+ * winK, winV, coefK, coefV and t_len are updated in place. */
 int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new,
                          const void *q, int batch, float *coefK, float *coefV, void *winK,
                          void *winV, int32_t *t_len, float scale, void *out, void *stream);
@@ -317,9 +334,10 @@ int faedkv_device_status(faedkv_ctx *ctx, void *stream);
  * Same arguments, layouts and result as faedkv_decode_attn() (float32
  * kernels); kv_dtype is the faedkv_dtype of q and out.  Sizes whose
  * intermediates, about 4*batch*HQP*(n_dft + 4*n_bins + n_dft/32) bytes with
- * HQP = n_q_heads rounded up to 32, exceed the array are refused with
- * FAEDKV_ERR_SHAPE before anything is launched.  On any failure a text is
- * written to err_msg (host, err_len bytes; may be NULL).
+ * HQP = n_q_heads rounded up to 32, exceed the array, and sizes with
+ * batch * n_kv_heads or batch * HQP / 32 above 65535 (a grid dimension), are
+ * refused with FAEDKV_ERR_SHAPE before anything is launched.  On any failure a
+ * text is written to err_msg (host, err_len bytes; may be NULL).
  *
  * All calls share the one array, which keeps the previous call's contents.
  * Nothing in it needs to start at zero, so nothing is cleared; but calls that

@@ -220,7 +220,8 @@ void orc_attention_dense(const double *q, int G, const double *Kt, const double 
         for (int c = 0; c < d; ++c) {
             double acc = 0.0;
             for (int n = 0; n < L; ++n) acc += s[n] * Vt[(size_t)n * d + c];
-            out[(size_t)g * d + c] = acc / den;
+            /* L = 0: Eq. 3 sums over no token at all; the empty sum is read as the zero vector */
+            out[(size_t)g * d + c] = L > 0 ? acc / den : 0.0;
         }
     }
     free(s);

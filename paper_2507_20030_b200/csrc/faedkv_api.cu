@@ -69,6 +69,7 @@ struct FftScratch {
 struct faedkv_ctx {
     faedkv_config cfg;
     int device = 0;
+    int n_sm = 1;  // multiprocessors of the device (grid sizing)
     int gq = 1;    // query heads per kv head
     int hqp = 32;  // n_q_heads rounded up to a multiple of 32
     int max_M = 0;
@@ -151,7 +152,7 @@ int launch_check(faedkv_ctx *ctx, const char *what) {
 int out_slices(const faedkv_ctx *ctx, int batch, int M) {
     // enough CTAs to fill the GPU twice over, at least 64 bins per slice
     const int units = batch * ctx->cfg.n_kv_heads;
-    int s = (2 * 148 + units - 1) / units;
+    int s = (2 * ctx->n_sm + units - 1) / units;
     int cap = (M + 63) / 64;
     if (s > cap) s = cap;
     if (s < 1) s = 1;
@@ -195,9 +196,9 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             CUDA_TRY(ctx, cudaMalloc(&ctx->Qf, B * 2 * (size_t)M * HQP * sizeof(float)));
             CUDA_TRY(ctx, cudaMalloc(&ctx->Pf, B * 2 * (size_t)M * HQP * sizeof(float)));
         }
-        // the slice count never exceeds 2*148 (units >= 1), nor ceil(M/64)
+        // the slice count never exceeds twice the SM count (units >= 1), nor ceil(M/64)
         int cap = (M + 63) / 64;
-        if (cap > 2 * 148) cap = 2 * 148;
+        if (cap > 2 * ctx->n_sm) cap = 2 * ctx->n_sm;
         ctx->out_slices_cap = cap;
         CUDA_TRY(ctx, cudaMalloc(&ctx->partial, B * c.n_kv_heads * (size_t)cap * ctx->gq * kHeadDim * sizeof(float)));
         ctx->max_M = M;
@@ -365,7 +366,7 @@ int launch_attn_tc(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const flo
     const int Gtot = (n_cols + 63) / 64 * 64;
     const int ncols = (Gtot % 256 == 0) ? 256 : (Gtot % 128 == 0) ? 128 : 64;
     const int col_blocks = Gtot / ncols;
-    constexpr int KB = 16 / GQ;
+    constexpr int KB = attn_bins_per_warp(GQ);
     // (1) scaled query spectrum in f16
     {
         dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
@@ -383,7 +384,7 @@ int launch_attn_tc(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const flo
         a.bins = p.d_bins; a.tab = p.d_tab; a.t_len = t_len; a.M = M; a.P = (uint32_t)P; a.Lrows = P;
         a.S = t.S; a.tile_max = t.tile_max; a.Gtot = Gtot; a.HQ = HQ; a.n_seq_cols = n_cols; a.status = ctx->dev_status;
         const int tiles2 = (P + 255) / 256;
-        const bool two = tiles2 * col_blocks >= 148;
+        const bool two = tiles2 * col_blocks >= ctx->n_sm;
         dim3 grid(two ? tiles2 : (P + 127) / 128, col_blocks);
         int r;
         if (ncols == 256) r = two ? launch_idft<256, 2, 1>(ctx, mq, mq, a, grid, st) : launch_idft<256, 1, 1>(ctx, mq, mq, a, grid, st);
@@ -404,7 +405,7 @@ int launch_attn_tc(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const flo
     }
     // (4) probability spectrum, positions split over CTAs
     const int bin_tiles = (M + 127) / 128;
-    int splits = (2 * 148 + bin_tiles * col_blocks - 1) / (bin_tiles * col_blocks);
+    int splits = (2 * ctx->n_sm + bin_tiles * col_blocks - 1) / (bin_tiles * col_blocks);
     if (splits > kSplitsCap) splits = kSplitsCap;
     if (splits > (P + 511) / 512) splits = (P + 511) / 512;
     if (splits < 1) splits = 1;
@@ -492,8 +493,8 @@ int launch_reconstruct_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const flo
         const int uc = units - u0 < f.recon_units ? units - u0 : f.recon_units;
         const fft::Geometry g = fft::make_geometry(c.n_dft, uc * kHeadDim);
         const int col_blocks = g.Gp / fft::kCW;
-        const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks));
-        const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks));
+        const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks, ctx->n_sm));
+        const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks, ctx->n_sm));
         int rc = FAEDKV_ERR_UNSUPPORTED;
         {
             const dim3 grid(g.N2 >> lgKT, col_blocks);
@@ -545,8 +546,8 @@ int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x
         const int uc = units - u0 < per ? units - u0 : per;
         const fft::Geometry g = fft::make_geometry(c.n_dft, uc * kHeadDim);
         const int col_blocks = g.Gp / fft::kCW;
-        const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks));
-        const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks));
+        const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks, ctx->n_sm));
+        const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks, ctx->n_sm));
         int rc = FAEDKV_ERR_UNSUPPORTED;
         {
             const dim3 grid(g.N1 >> lgMT, col_blocks);
@@ -603,20 +604,22 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
     const int H = c.n_kv_heads, HQ = c.n_q_heads, M = p.M, P = c.n_dft;
     const fft::Geometry g = fft::make_geometry(P, batch * HQ);
     const int col_blocks = g.Gp / fft::kCW;
-    const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks));
-    const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks));
-    constexpr int KB = 16 / GQ;
+    const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks, ctx->n_sm));
+    const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks, ctx->n_sm));
+    constexpr int KB = attn_bins_per_warp(GQ);
     // step (5) for the sequences [b0, b1) on stream s
     auto launch_out = [&](int b0, int b1, cudaStream_t s) -> int {
         const int nb = b1 - b0;
         const int slices = out_slices(ctx, nb, M);
+        // one stride for every launch of the call, whatever its own slice count: runs never share a partial slot
+        const int slice_stride = ctx->out_slices_cap;
         const int per = (M + slices - 1) / slices;
         dim3 grid(slices, nb * H);
         launch_pdl(k_attn_out_fft<TQ, GQ, APPEND>, grid, dim3(kAttnWarps * 32), 0, s,
                    coefV, static_cast<const TQ *>(foldV), t_len, f.Zf, f.colsum, p.d_bins, ctx->partial, f.tickets,
                    static_cast<TQ *>(out), M, H, HQ, g, per, 1.0f / (float)P, fold, n_extra ? f.o_win : nullptr, counts_new ? 1 : 0,
                    windowed ? WindowArgs{winK, winV, k_new, v_new, S, R, D, Rc, 0.f, nullptr, nullptr, nullptr} : WindowArgs{},
-                   ctx->use_col ? f.Wg : nullptr, b0 * H, batch * H);
+                   ctx->use_col ? f.Wg : nullptr, b0 * H, batch * H, slice_stride);
         return launch_check(ctx, "k_attn_out_fft");
     };
     if (n_extra) {
@@ -651,7 +654,7 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
         // pass over C_V streams while the second run's columns are still being transformed.
         const int lgn = g.lgN1 + g.lgN2;
         const int ctas_per_sm = lgn >= 13 ? 2 : (lgn == 12 ? 3 : (lgn == 11 ? 7 : 16));   // registers / shared memory
-        const int b_cut = (batch >= 2 && batch * HQ > ctas_per_sm * 148) ? batch / 2 : batch;
+        const int b_cut = (batch >= 2 && batch * HQ > ctas_per_sm * ctx->n_sm) ? batch / 2 : batch;
         auto launch_col = [&](int b0, int b1, cudaStream_t s) -> int {
             int rcc = FAEDKV_ERR_UNSUPPORTED;
 #define CALL(LG)                                                                                         \
@@ -742,10 +745,14 @@ int dispatch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const 
     switch (ctx->gq) {
         case 1: return launch_attn_fft<TQ, 1, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
         case 2: return launch_attn_fft<TQ, 2, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+        case 3: return launch_attn_fft<TQ, 3, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
         case 4: return launch_attn_fft<TQ, 4, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+        case 5: return launch_attn_fft<TQ, 5, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+        case 6: return launch_attn_fft<TQ, 6, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
+        case 7: return launch_attn_fft<TQ, 7, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
         case 8: return launch_attn_fft<TQ, 8, APPEND>(ctx, p, q, k_new, v_new, coefK, coefV, t_len, batch, scale, out, st, winK, winV);
     }
-    return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be 1, 2, 4 or 8");
+    return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be between 1 and 8");
 }
 
 __global__ void k_set_tlen(int32_t *t_len, int batch, int T) {
@@ -795,7 +802,7 @@ int launch_attn(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const float 
     const faedkv_config &c = ctx->cfg;
     const int H = c.n_kv_heads, HQ = c.n_q_heads, HQP = ctx->hqp, M = p.M, P = c.n_dft;
     const int col_blocks = HQP / 32;
-    constexpr int KB = 16 / GQ;
+    constexpr int KB = attn_bins_per_warp(GQ);
     // (1) query spectrum
     {
         dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), batch * H);
@@ -884,17 +891,25 @@ int dispatch_attn(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const floa
         switch (ctx->gq) {
             case 1: return launch_attn_tc<TQ, 1>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
             case 2: return launch_attn_tc<TQ, 2>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+            case 3: return launch_attn_tc<TQ, 3>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
             case 4: return launch_attn_tc<TQ, 4>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+            case 5: return launch_attn_tc<TQ, 5>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+            case 6: return launch_attn_tc<TQ, 6>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+            case 7: return launch_attn_tc<TQ, 7>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
             case 8: return launch_attn_tc<TQ, 8>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
         }
     }
     switch (ctx->gq) {
         case 1: return launch_attn<TQ, 1>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
         case 2: return launch_attn<TQ, 2>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 3: return launch_attn<TQ, 3>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
         case 4: return launch_attn<TQ, 4>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 5: return launch_attn<TQ, 5>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 6: return launch_attn<TQ, 6>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 7: return launch_attn<TQ, 7>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
         case 8: return launch_attn<TQ, 8>(ctx, p, q, coefK, coefV, t_len, batch, scale, out, st);
     }
-    return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be 1, 2, 4 or 8");
+    return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be between 1 and 8");
 }
 
 }  // namespace
@@ -920,7 +935,10 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
     if (cfg->head_dim != kHeadDim) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FAEDKV_ERR_UNSUPPORTED;
     const int gq = cfg->n_q_heads / cfg->n_kv_heads;
-    if (gq != 1 && gq != 2 && gq != 4 && gq != 8) return FAEDKV_ERR_UNSUPPORTED;
+    if (gq < 1 || gq > 8) return FAEDKV_ERR_UNSUPPORTED;
+    // units and column blocks index gridDim.y
+    if ((long long)cfg->max_batch * cfg->n_kv_heads > 65535 || (long long)cfg->max_batch * cfg->n_q_heads / 16 > 65535)
+        return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->prefill_mode == FAEDKV_PREFILL_UMMA && cfg->kv_dtype != FAEDKV_BF16) return FAEDKV_ERR_UNSUPPORTED;
 
     faedkv_ctx *ctx = new (std::nothrow) faedkv_ctx();
@@ -940,6 +958,7 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
                                         (cfg->prefill_mode == FAEDKV_PREFILL_AUTO && cfg->kv_dtype == FAEDKV_F32));
     ctx->plans.resize(cfg->n_layers);
     if (cudaGetDevice(&ctx->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess || ctx->n_sm < 1 ||
         cudaMalloc(&ctx->tick, sizeof(unsigned int) * (cfg->n_layers + 1)) != cudaSuccess ||
         cudaMemset(ctx->tick, 0, sizeof(unsigned int) * (cfg->n_layers + 1)) != cudaSuccess) {
         cudaGetLastError();
@@ -1245,9 +1264,9 @@ int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const vo
         // work items (sequence, 32 bins, share of the 2H planes); the planes are split until the items fill the SMs
         const int n_groups = (p->M + kFoldGroup - 1) / kFoldGroup;
         int splits = 1;
-        while (splits < 2 * c.n_kv_heads && batch * n_groups * splits < 4 * 148) splits *= 2;
+        while (splits < 2 * c.n_kv_heads && batch * n_groups * splits < 4 * ctx->n_sm) splits *= 2;
         const int n_items = batch * n_groups * splits;
-        const dim3 grid(n_items < 4 * 148 ? n_items : 4 * 148);
+        const dim3 grid(n_items < 4 * ctx->n_sm ? n_items : 4 * ctx->n_sm);
         const size_t smem = block_fold_smem(D);
         if (c.kv_dtype == FAEDKV_BF16) {
             if (int r = fft_opt_in(ctx, k_block_fold<__nv_bfloat16>, smem, ctx->fs.attr_mask[9], 0)) return r;

@@ -13,13 +13,14 @@
 //
 // Consequences of the fixed array:
 //  * every GPU that loads the library holds kStaticScratchBytes until exit;
-//  * problem sizes whose intermediates do not fit are rejected with
-//    FAEDKV_ERR_SHAPE before anything is launched;
+//  * problem sizes whose intermediates do not fit the array, or whose launch grids would exceed the
+//    device's grid limits, are rejected with FAEDKV_ERR_SHAPE before anything is launched;
 //  * all calls share the array and it keeps whatever the last call left in it.
-//    Nothing in it has to start at zero (each region is fully written before it
-//    is read; padded query-head columns are never read back), so no clearing is
-//    done; but two calls that overlap on the GPU (different streams, or the same
-//    call from two threads) race on it.  Serialise them.
+//    Nothing in it has to start at zero: each region's real columns are fully written before they
+//    are read.  The padding columns (query heads rounded up to 32) are read by the two transforms with
+//    whatever an earlier call left there, but columns are independent and a padding column never
+//    feeds an output.  So no clearing is done; but two calls that overlap on the GPU (different
+//    streams, or the same call from two threads) race on the array.  Serialise them.
 //  * the first call on each device looks up the array's device address
 //    (cudaGetSymbolAddress); make that first call before any stream capture.
 #include <cstdio>
@@ -28,9 +29,6 @@
 #include "../../include/faedkv.h"
 #include "common.cuh"
 #include "k_attn.cuh"
-// k_dft_simt.cuh defines one non-template kernel; give this translation unit's copy its own name so the
-// two object files link without touching the shared header.
-#define k_colmax k_colmax_static_tu
 #include "k_dft_simt.cuh"
 
 using namespace faedkv;
@@ -46,6 +44,7 @@ static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
 
 std::mutex g_mutex;
 float *g_scratch_addr[kMaxDevices] = {nullptr};
+int g_sm_count[kMaxDevices] = {0};
 // Where the current call wants its error text (caller's buffer; may be absent).
 thread_local char *g_err = nullptr;
 thread_local size_t g_err_len = 0;
@@ -60,8 +59,9 @@ int fail(int code, const char *msg) {
     return code;
 }
 
-// Device address of the scratch array on the current device; resolved once per device.
-int scratch_for_current_device(float **out) {
+// Device address of the scratch array on the current device (and the device's SM count, for grid sizing);
+// resolved once per device.
+int scratch_for_current_device(float **out, int *n_sm) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return fail(FAEDKV_ERR_CUDA, "cudaGetDevice failed");
     if (dev < 0 || dev >= kMaxDevices) return fail(FAEDKV_ERR_UNSUPPORTED, "device ordinal beyond the table of scratch addresses");
@@ -73,23 +73,35 @@ int scratch_for_current_device(float **out) {
             set_err("cudaGetSymbolAddress(static scratch) failed: %s", cudaGetErrorString(e));
             return FAEDKV_ERR_CUDA;
         }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+            return fail(FAEDKV_ERR_CUDA, "cannot read the device's multiprocessor count");
+        g_sm_count[dev] = sms;
         g_scratch_addr[dev] = p;
     }
     *out = g_scratch_addr[dev];
+    *n_sm = g_sm_count[dev];
     return FAEDKV_OK;
 }
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 template <typename TQ, int GQ>
-int run(float *scratch, int P, int H, int HQ, const int32_t *bins, int M, const void *q, const float *coefK,
+int run(float *scratch, int n_sm, int P, int H, int HQ, const int32_t *bins, int M, const void *q, const float *coefK,
         const float *coefV, const int32_t *t_len, int batch, float scale, void *out, cudaStream_t st) {
     const int HQP = (HQ + 31) / 32 * 32, col_blocks = HQP / 32;
     const int n_tiles = (P + kTilePos - 1) / kTilePos;
     const int units = batch * H;
-    int slices = (2 * 148 + units - 1) / units;
+    int slices = (2 * n_sm + units - 1) / units;
     if (slices > (M + 63) / 64) slices = (M + 63) / 64;
     if (slices < 1) slices = 1;
+    // every launch below puts units or batch * col_blocks in gridDim.y
+    constexpr long long kMaxGridY = 65535;
+    if ((long long)units > kMaxGridY || (long long)batch * col_blocks > kMaxGridY) {
+        set_err("batch * n_kv_heads = %d (or batch * column blocks = %lld) exceeds the grid limit %lld", units,
+                (long long)batch * col_blocks, kMaxGridY);
+        return FAEDKV_ERR_SHAPE;
+    }
     // carve the array (64-float granules keep every region 256-byte aligned)
     size_t off = 0;
     auto take = [&](size_t n) { float *p = scratch + off; off += round_up(n, 64); return p; };
@@ -104,7 +116,7 @@ int run(float *scratch, int P, int H, int HQ, const int32_t *bins, int M, const 
                 off * sizeof(float), kStaticScratchBytes);
         return FAEDKV_ERR_SHAPE;
     }
-    constexpr int KB = 16 / GQ;
+    constexpr int KB = attn_bins_per_warp(GQ);
     {
         dim3 grid((M + kAttnWarps * KB - 1) / (kAttnWarps * KB), units);
         k_attn_qf<TQ, GQ><<<grid, kAttnWarps * 32, 0, st>>>(static_cast<const TQ *>(q), coefK, Qf, M, H, HQ, HQP);
@@ -143,16 +155,20 @@ int run(float *scratch, int P, int H, int HQ, const int32_t *bins, int M, const 
 }
 
 template <typename TQ>
-int dispatch(int gq, float *scratch, int P, int H, int HQ, const int32_t *bins, int M, const void *q,
+int dispatch(int gq, float *scratch, int n_sm, int P, int H, int HQ, const int32_t *bins, int M, const void *q,
              const float *coefK, const float *coefV, const int32_t *t_len, int batch, float scale, void *out,
              cudaStream_t st) {
     switch (gq) {
-        case 1: return run<TQ, 1>(scratch, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
-        case 2: return run<TQ, 2>(scratch, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
-        case 4: return run<TQ, 4>(scratch, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
-        case 8: return run<TQ, 8>(scratch, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 1: return run<TQ, 1>(scratch, n_sm, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 2: return run<TQ, 2>(scratch, n_sm, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 3: return run<TQ, 3>(scratch, n_sm, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 4: return run<TQ, 4>(scratch, n_sm, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 5: return run<TQ, 5>(scratch, n_sm, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 6: return run<TQ, 6>(scratch, n_sm, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 7: return run<TQ, 7>(scratch, n_sm, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
+        case 8: return run<TQ, 8>(scratch, n_sm, P, H, HQ, bins, M, q, coefK, coefV, t_len, batch, scale, out, st);
     }
-    return fail(FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be 1, 2, 4 or 8");
+    return fail(FAEDKV_ERR_UNSUPPORTED, "query heads per kv head must be between 1 and 8");
 }
 
 }  // namespace
@@ -180,13 +196,14 @@ int faedkv_decode_attn_static(int n_dft, int n_kv_heads, int n_q_heads, int kv_d
         return fail(FAEDKV_ERR_ALIGN, "bins / t_len not 4-byte aligned");
     if (scale == 0.0f) scale = 1.0f / sqrtf((float)kHeadDim);
     float *scratch = nullptr;
-    if (int r = scratch_for_current_device(&scratch)) return r;
+    int n_sm = 0;
+    if (int r = scratch_for_current_device(&scratch, &n_sm)) return r;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int gq = n_q_heads / n_kv_heads;
     if (kv_dtype == FAEDKV_BF16)
-        return dispatch<__nv_bfloat16>(gq, scratch, n_dft, n_kv_heads, n_q_heads, bins, n_bins, q, coefK, coefV, t_len,
+        return dispatch<__nv_bfloat16>(gq, scratch, n_sm, n_dft, n_kv_heads, n_q_heads, bins, n_bins, q, coefK, coefV, t_len,
                                        batch, scale, out, st);
-    return dispatch<float>(gq, scratch, n_dft, n_kv_heads, n_q_heads, bins, n_bins, q, coefK, coefV, t_len, batch,
+    return dispatch<float>(gq, scratch, n_sm, n_dft, n_kv_heads, n_q_heads, bins, n_bins, q, coefK, coefV, t_len, batch,
                            scale, out, st);
 }
 

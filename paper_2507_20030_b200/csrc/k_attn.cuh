@@ -36,12 +36,16 @@ __device__ __forceinline__ float warp_transpose_reduce32(float (&v)[32], int lan
     return v[0];
 }
 
-// (1) grid = (ceil(M / (8 * KB)), batch * H); block = 256; KB = 16 / GQ bins per warp.
+// Bins a warp of the C_K pass takes: KB bins x 2 planes x GQ query heads are the (at most 32) dot products
+// that one transpose-reduce finishes; any GQ from 1 to 8 (with GQ = 3, 5, 6, 7 a few of the 32 slots stay empty).
+__host__ __device__ constexpr int attn_bins_per_warp(int GQ) { return 16 / GQ; }
+
+// (1) grid = (ceil(M / (8 * KB)), batch * H); block = 256; KB = attn_bins_per_warp(GQ).
 template <typename TQ, int GQ>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 k_attn_qf(const TQ *__restrict__ q, const float *__restrict__ coefK, float *__restrict__ Qf,
           int M, int H, int HQ, int HQP) {
-    constexpr int KB = 16 / GQ;  // bins per warp: KB * 2 planes * GQ heads = 32 values
+    constexpr int KB = attn_bins_per_warp(GQ);  // KB * 2 planes * GQ heads <= 32 values
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
     const int k0 = (blockIdx.x * kAttnWarps + warp) * KB;
@@ -63,6 +67,8 @@ k_attn_qf(const TQ *__restrict__ q, const float *__restrict__ coefK, float *__re
         }
     float v[32];
 #pragma unroll
+    for (int i = KB * 2 * GQ; i < 32; ++i) v[i] = 0.f;
+#pragma unroll
     for (int kk = 0; kk < KB; ++kk)
 #pragma unroll
         for (int pl = 0; pl < 2; ++pl)
@@ -73,7 +79,7 @@ k_attn_qf(const TQ *__restrict__ q, const float *__restrict__ coefK, float *__re
             }
     const float tot = warp_transpose_reduce32(v, lane);
     const int kk = lane / (2 * GQ), pl = (lane / GQ) & 1, g = lane % GQ;
-    if (k0 + kk < M)
+    if (kk < KB && k0 + kk < M)
         Qf[(((size_t)b * 2 + pl) * M + (k0 + kk)) * HQP + h * GQ + g] = tot;
 }
 

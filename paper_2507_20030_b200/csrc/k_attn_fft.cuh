@@ -24,13 +24,13 @@
 namespace faedkv {
 
 // ---- (1) ------------------------------------------------------------------------------------------
-// grid = (ceil(M / (8 * KB)), batch * H); block = 256; KB = 16 / GQ bins per warp.
+// grid = (ceil(M / (8 * KB)), batch * H); block = 256; KB = attn_bins_per_warp(GQ) bins per warp.
 template <typename TQ, int GQ, bool APPEND>
 __global__ void __launch_bounds__(kAttnWarps * 32, 3)
 k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restrict__ k_new,
           const int32_t *__restrict__ t_len, const int32_t *__restrict__ bins, float2 *__restrict__ Qs,
           int M, int H, int HQ, int Gp, uint32_t P, float scale_over_P, FoldSrc fold, int col_major) {
-    constexpr int KB = 16 / GQ;
+    constexpr int KB = attn_bins_per_warp(GQ);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
@@ -56,6 +56,8 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
     constexpr int GB = KB < 4 ? KB : 4;
     float v[32];
 #pragma unroll
+    for (int i = KB * 2 * GQ; i < 32; ++i) v[i] = 0.f;
+#pragma unroll
     for (int g0 = 0; g0 < KB; g0 += GB) {
         float4 row[GB][2];
 #pragma unroll
@@ -63,12 +65,12 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
 #pragma unroll
             for (int pl = 0; pl < 2; ++pl) {
                 row[kk][pl] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (k0 + g0 + kk < M) row[kk][pl] = ld_stream(base + pl * plane + (size_t)(k0 + g0 + kk) * kHeadDim + lane * 4);
+                if (g0 + kk < KB && k0 + g0 + kk < M) row[kk][pl] = ld_stream(base + pl * plane + (size_t)(k0 + g0 + kk) * kHeadDim + lane * 4);
             }
         if (APPEND) {
 #pragma unroll
             for (int kk = 0; kk < GB; ++kk) {
-                if (k0 + g0 + kk >= M) continue;
+                if (g0 + kk >= KB || k0 + g0 + kk >= M) continue;
                 float c, sn;
                 twiddle(phase_mod((uint32_t)bins[k0 + g0 + kk], t, P), P, c, sn);
                 float4 &re = row[kk][0], &im = row[kk][1];
@@ -87,13 +89,14 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
             for (int pl = 0; pl < 2; ++pl)
 #pragma unroll
                 for (int g = 0; g < GQ; ++g) {
+                    if (g0 + kk >= KB) continue;       // KB need not be a multiple of the group size
                     const float4 r = row[kk][pl];
                     v[((g0 + kk) * 2 + pl) * GQ + g] = r.x * qv[g].x + r.y * qv[g].y + r.z * qv[g].z + r.w * qv[g].w;
                 }
     }
     const float tot = warp_transpose_reduce32(v, lane);
     const int kk = lane / (2 * GQ), pl = (lane / GQ) & 1, g = lane % GQ;
-    if (k0 + kk < M) {
+    if (kk < KB && k0 + kk < M) {
         const uint32_t bin = (uint32_t)bins[k0 + kk];
         // bins 0 and P/2 are their own mirrors: only their real part enters a real signal
         const bool self_conj = bin == 0u || 2u * bin == P;
@@ -349,6 +352,9 @@ inline size_t afft_smem_fwd_b(int lg, int lgKT, int lgMT) {
 // formula; one thread per bin) into shared memory, then the warps stream the coefficient rows, four
 // bins per warp in flight.  The last CTA of a (sequence, kv head) to finish sums the slice partials in
 // a fixed order, divides by P * colsum and writes the output rows.
+// The partials of unit bh sit at partial[bh * slice_stride + slice]: the stride is the same for every launch of
+// one call (a call cut into two runs of sequences launches twice, possibly with different slice counts, and
+// the runs overlap in time), so no two units ever share a slot.
 // grid = (slices, batch * H); block = 256.
 constexpr int kOutChunk = 256;
 
@@ -359,7 +365,7 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
                float *__restrict__ partial, unsigned int *__restrict__ tickets, TQ *__restrict__ out,
                int M, int H, int HQ, fft::Geometry g, int bins_per_slice, float inv_P, FoldSrc fold,
                const float *__restrict__ o_win, int bump, WindowArgs commit, const float2 *__restrict__ Wg,
-               int bh0, int n_units) {
+               int bh0, int n_units, int slice_stride) {
     using namespace fft;
     // the weights of a chunk and the final cross-warp reduction share one buffer
     constexpr size_t kWgtBytes = (size_t)kOutChunk * GQ * sizeof(float2) + (APPEND ? kOutChunk * sizeof(float2) : 0);
@@ -467,7 +473,7 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
         float s = 0.f;
 #pragma unroll
         for (int w = 0; w < kAttnWarps; ++w) s += red[w][q][c];
-        partial[(((size_t)bh * gridDim.x + blockIdx.x) * GQ + q) * kHeadDim + c] = s;
+        partial[(((size_t)bh * slice_stride + blockIdx.x) * GQ + q) * kHeadDim + c] = s;
     }
     // last CTA of this (sequence, kv head): reduce the slices in a fixed order
     __threadfence();
@@ -484,11 +490,13 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
             const int q = e / kHeadDim, c = e % kHeadDim;
             float s = 0.f;
             for (int sl = 0; sl < (int)gridDim.x; ++sl)
-                s += __ldcg(partial + (((size_t)bh * gridDim.x + sl) * GQ + q) * kHeadDim + c);
+                s += __ldcg(partial + (((size_t)bh * slice_stride + sl) * GQ + q) * kHeadDim + c);
             s *= inv_P;
             // the sink + recent window's share of the same softmax (its factor sits behind the normalisers)
             if (o_win != nullptr) s = fmaf(o_win[(size_t)(gcol + q) * kHeadDim + c], colsum[g.Gp + gcol + q], s);
-            store1(out + (size_t)(gcol + q) * kHeadDim + c, s / colsum[gcol + q]);
+            // a sequence with no visible token (t_len = 0 and no window) has an empty softmax: its output is zero
+            const float den = colsum[gcol + q];
+            store1(out + (size_t)(gcol + q) * kHeadDim + c, den > 0.f ? s / den : 0.f);
         }
         if (bump) {
             // every CTA of this sequence has read t_len (and the token it folds) before taking its ticket; the

@@ -20,7 +20,7 @@ template <typename TQ, int GQ>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 k_attn_qf16(const TQ *__restrict__ q, const float *__restrict__ coefK, const int32_t *__restrict__ bins,
             __half *__restrict__ Qf16, int M, int H, int HQ, int Gtot, uint32_t P, float scale_over_P) {
-    constexpr int KB = 16 / GQ;
+    constexpr int KB = attn_bins_per_warp(GQ);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bh = blockIdx.y, b = bh / H, h = bh % H;
     const int k0 = (blockIdx.x * kAttnWarps + warp) * KB;
@@ -40,6 +40,8 @@ k_attn_qf16(const TQ *__restrict__ q, const float *__restrict__ coefK, const int
         }
     float v[32];
 #pragma unroll
+    for (int i = KB * 2 * GQ; i < 32; ++i) v[i] = 0.f;
+#pragma unroll
     for (int kk = 0; kk < KB; ++kk)
 #pragma unroll
         for (int pl = 0; pl < 2; ++pl)
@@ -50,7 +52,7 @@ k_attn_qf16(const TQ *__restrict__ q, const float *__restrict__ coefK, const int
             }
     const float tot = warp_transpose_reduce32(v, lane);
     const int kk = lane / (2 * GQ), pl = (lane / GQ) & 1, g = lane % GQ;
-    if (k0 + kk < M) {
+    if (kk < KB && k0 + kk < M) {
         const float w = hermitian_weight((uint32_t)bins[k0 + kk], P) * scale_over_P;
         Qf16[((size_t)pl * M + (k0 + kk)) * Gtot + b * HQ + h * GQ + g] = __float2half_rn(tot * w);
     }
@@ -367,7 +369,8 @@ __global__ void k_attn_out_reduce2(const float *__restrict__ partial, const floa
     float s = 0.f;
     for (int sl = 0; sl < slices; ++sl) s += partial[(((size_t)bh * slices + sl) * GQ + g) * kHeadDim + c];
     // flat query-head index bh * GQ + g equals the column index sequence * HQ + head
-    store1(out + ((size_t)bh * GQ + g) * kHeadDim + c, s * inv_P / colsum[bh * GQ + g]);
+    const float den = colsum[bh * GQ + g];          // zero only when the sequence has no token: output zero
+    store1(out + ((size_t)bh * GQ + g) * kHeadDim + c, den > 0.f ? s * inv_P / den : 0.f);
 }
 
 }  // namespace faedkv

@@ -150,7 +150,7 @@ k_dft_forward_simt(DftUnitArgs a, const int32_t *__restrict__ bins, int M, uint3
 #pragma unroll
         for (int q = 0; q < CPT; ++q) {
             float inv = 1.f;
-            if (SOFTMAX_IN) inv = 1.f / colsum[q];
+            if (SOFTMAX_IN) inv = colsum[q] > 0.f ? 1.f / colsum[q] : 0.f;   // no live row: the spectrum of nothing is zero
             const size_t o = (size_t)k * a.y_row + lane * CPT + q;
             float re = accre[i][q] * inv, im = sgn * accim[i][q] * inv;
             if (accumulate) { re += yre[o]; im += yim[o]; }
@@ -298,8 +298,8 @@ k_dft_inverse_simt(DftUnitArgs a, const int32_t *__restrict__ bins, int M, uint3
 }
 
 // Column maxima over the row tiles: colmax[u*ncol + c] = max_tile tile_max[u][tile][c],
-// u = sequence * col_blocks + block.
-__global__ void k_colmax(const float *__restrict__ tile_max, int n_tiles, int ncol,
+// u = sequence * col_blocks + block.  (static: this header is compiled into more than one translation unit.)
+static __global__ void k_colmax(const float *__restrict__ tile_max, int n_tiles, int ncol,
                          float *__restrict__ colmax) {
     const int u = blockIdx.x;
     for (int c = threadIdx.x; c < ncol; c += blockDim.x) {

@@ -56,11 +56,11 @@ inline Geometry make_geometry(int P, int G) {
 inline bool supported(int P) { return P >= 64 && P <= (1 << 19) && (P & (P - 1)) == 0; }
 
 // How many transforms of a pass one CTA takes (a power of two): fill the tile, but keep at least
-// ~2 CTAs per SM in the grid when the problem allows.
-inline int transforms_per_cta(int rows, int n_transforms, int col_blocks) {
+// ~2 CTAs per SM (n_sm of them on the device) in the grid when the problem allows.
+inline int transforms_per_cta(int rows, int n_transforms, int col_blocks, int n_sm) {
     int kt = kTileMax / (rows * kCW);
     if (kt < 1) kt = 1;
-    while (kt > 1 && (kt > n_transforms || (n_transforms / kt) * col_blocks < 2 * 148)) kt >>= 1;
+    while (kt > 1 && (kt > n_transforms || (n_transforms / kt) * col_blocks < 2 * n_sm)) kt >>= 1;
     return kt;
 }
 

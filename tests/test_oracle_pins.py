@@ -294,6 +294,22 @@ def test_all_bins_attention_is_textbook(oracle, P, t):
     np.testing.assert_allclose(out2, _textbook_attention(q, K, V, 0.37), atol=1e-12)
 
 
+def test_attention_over_no_token_is_zero(oracle):
+    """L = 0: Eq. 3 has no token to sum over; the reading taken is the empty sum, a zero vector (never NaN),
+    and one token gives that token's value row whatever the query."""
+    P, d, G = 16, 8, 3
+    rng = _rng(5)
+    q = rng.standard_normal((G, d))
+    bins = _all_bins(P)
+    V = rng.standard_normal((1, d))
+    kr, ki = oracle.compress(rng.standard_normal((1, d)), P, bins)
+    vr, vi = oracle.compress(V, P, bins)
+    out0 = oracle.decode_attn(q, kr, ki, vr, vi, P, bins, 0)
+    assert out0.shape == (G, d) and not out0.any()
+    out1 = oracle.decode_attn(q, kr, ki, vr, vi, P, bins, 1)
+    np.testing.assert_allclose(out1, np.broadcast_to(V[0], (G, d)), atol=1e-12)
+
+
 # ----------------------------------------------------------------- P12: frequency-domain attention formula
 def test_frequency_domain_attention_identity(oracle):
     """softmax(q K~^T) V~ can be evaluated without materialising K~, V~:
