@@ -104,6 +104,10 @@ typedef struct {
                           uses 50); n_sink + n_recent <= 1024                        */
     int n_defer;       /* D: 0 or 1 = the paper's step, one token folded per step (Eq. 12);
                           2 .. 128 = block-deferred fold, see the window section       */
+    int recon_engine;  /* FFT-shaped reconstruction: 0 = default (one persistent kernel that runs both
+                          passes for P <= 2^15, the two-kernel engine above that), 1 = always the
+                          two-kernel engine (one launch per pass and group of units), 2 = the
+                          persistent kernel wherever it exists (P <= 2^17)                    */
 } faedkv_config;
 
 /* Create a context on the CURRENT CUDA device.  Allocates only a few counters; the scratch area

@@ -46,7 +46,7 @@ class FaedkvError(RuntimeError):
 class Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in (
         "n_layers", "n_kv_heads", "n_q_heads", "head_dim", "n_dft", "max_batch", "kv_dtype",
-        "prefill_mode", "twiddle_terms", "decode_mode", "n_sink", "n_recent", "n_defer")]
+        "prefill_mode", "twiddle_terms", "decode_mode", "n_sink", "n_recent", "n_defer", "recon_engine")]
 
 
 _lib = None
@@ -216,12 +216,13 @@ class Context:
     n_sink: int = 0
     n_recent: int = 0
     n_defer: int = 0
+    recon_engine: int = 0
 
     def __post_init__(self):
         self._lib = load()
         cfg = Config(self.n_layers, self.n_kv_heads, self.n_q_heads, self.head_dim, self.n_dft,
                      self.max_batch, self.kv_dtype, self.prefill_mode, self.twiddle_terms, self.decode_mode,
-                     self.n_sink, self.n_recent, self.n_defer)
+                     self.n_sink, self.n_recent, self.n_defer, self.recon_engine)
         h = _vp()
         rc = self._lib.faedkv_create(ctypes.byref(cfg), ctypes.byref(h))
         if rc != 0:

@@ -20,6 +20,7 @@
 #include "k_attn_fft.cuh"
 #include "k_attn_col.cuh"
 #include "k_recon_fft.cuh"
+#include "k_recon2.cuh"
 #include "k_prefill_fft.cuh"
 #include "k_ablate.cuh"
 #include "k_state.cuh"
@@ -59,6 +60,12 @@ struct FftScratch {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaStream_t side2 = nullptr;         // third stream: the second run of sequences of a call cut in two
     cudaEvent_t ev_cut = nullptr, ev_merge = nullptr;
+    // second reconstruction engine (one persistent kernel; P <= 2^17)
+    float2 *r2_tabP = nullptr, *r2_tabI = nullptr;
+    unsigned int *r2_sync = nullptr;      // ticket, exit counter, per-column-block pass counters; zero between calls
+    size_t yr_bytes = 0;                  // size of Yr
+    unsigned int r2_attr = 0;             // instances already opted in to large shared memory
+    int r2_ctas_per_sm[2][32] = {};       // occupancy of each instance (0 = not asked yet)
     unsigned int *tickets = nullptr;      // [max_batch * H + max_batch], zero between calls
     int max_M = 0;
     unsigned int attr_mask[11] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};  // per kernel: transform lengths already opted in to large shared memory
@@ -168,7 +175,7 @@ void free_scratch(faedkv_ctx *ctx) {
     cudaFree(t.cmax); cudaFree(t.psum); cudaFree(t.colsum); cudaFree(t.PfS);
     t = TcScratch();
     FftScratch &f = ctx->fs;
-    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.o_win); cudaFree(f.Wg); cudaFree(f.colE); cudaFree(f.colB); cudaFree(f.colP); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr);
+    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.o_win); cudaFree(f.Wg); cudaFree(f.colE); cudaFree(f.colB); cudaFree(f.colP); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr); cudaFree(f.r2_tabP); cudaFree(f.r2_tabI); cudaFree(f.r2_sync);
     if (f.side != nullptr) cudaStreamDestroy(f.side);
     if (f.ev_fork != nullptr) cudaEventDestroy(f.ev_fork);
     if (f.ev_join != nullptr) cudaEventDestroy(f.ev_join);
@@ -229,7 +236,17 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
             if (ru < 1) ru = 1;
             if (ru > (size_t)c.max_batch * c.n_kv_heads) ru = (size_t)c.max_batch * c.n_kv_heads;
             f.recon_units = (int)ru;
+            f.yr_bytes = ru * unit_bytes;
             CUDA_TRY(ctx, cudaMalloc(&f.Yr, ru * unit_bytes));
+            if (rfft2::supported(c.n_dft)) {
+                const size_t n_sync = 2 + 2 * (size_t)2 * c.max_batch * c.n_kv_heads * (kHeadDim / rfft2::kCW);
+                CUDA_TRY(ctx, cudaMalloc(&f.r2_tabP, ((size_t)g.N + 1) * sizeof(float2)));
+                CUDA_TRY(ctx, cudaMalloc(&f.r2_tabI, (size_t)g.N * sizeof(float2)));
+                CUDA_TRY(ctx, cudaMalloc(&f.r2_sync, n_sync * sizeof(unsigned int)));
+                CUDA_TRY(ctx, cudaMemset(f.r2_sync, 0, n_sync * sizeof(unsigned int)));
+                rfft2::k_recon2_tables<<<64, 256>>>(f.r2_tabP, f.r2_tabI, (uint32_t)c.n_dft, g.N2);
+                CUDA_TRY(ctx, cudaDeviceSynchronize());
+            }
             if (ctx->prefill_fft) CUDA_TRY(ctx, cudaMalloc(&f.Zr, ru * unit_bytes));
         }
         if (M > f.max_M) {
@@ -523,10 +540,81 @@ int launch_reconstruct_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const flo
     return FAEDKV_OK;
 }
 
+// Which reconstruction engine a call takes: the persistent one where it exists and is the faster of the two (measured:
+// 1.3 - 1.4x faster up to 128 x 128 points per channel, slower at 256-point passes, whose radix-16 x 16 butterflies
+// leave it three CTAs per SM), unless the configuration asks for the two-kernel engine.
+bool use_recon2(const faedkv_ctx *ctx) {
+    if (ctx->fs.r2_sync == nullptr || ctx->cfg.recon_engine == 1) return false;
+    if (ctx->cfg.recon_engine == 2) return true;
+    return ctx->cfg.n_dft <= (1 << 15);
+}
+
+// Second engine: both tensors, both passes, one persistent launch (k_recon2.cuh).
+template <int LG1, int LG2, typename TOut>
+int launch_recon2_t(faedkv_ctx *ctx, rfft2::Args &a, int inst, cudaStream_t st) {
+    FftScratch &f = ctx->fs;
+    constexpr size_t smem = rfft2::smem_bytes<LG1, LG2>();
+    constexpr int kind = sizeof(TOut) == 2 ? 0 : 1;
+    auto kernel = rfft2::k_recon2<LG1, LG2, TOut>;
+    const unsigned int bit = 1u << (inst + 16 * kind);
+    if (smem > 48 * 1024 && !(f.r2_attr & bit)) {
+        if (int r = opt_in_smem(ctx, kernel, (uint32_t)smem)) return r;
+        f.r2_attr |= bit;
+    }
+    int &occ = f.r2_ctas_per_sm[kind][inst];
+    if (occ == 0) {
+        CUDA_TRY(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kernel, rfft2::kThreads, smem));
+        if (occ < 1) return fail(ctx, FAEDKV_ERR_CUDA, "the reconstruction kernel does not fit an SM");
+    }
+    constexpr int nA = (1 << LG2) >> rfft2::lg_per_tile(LG1, LG2), nB = (1 << LG1) >> rfft2::lg_per_tile(LG2, LG1);
+    const int n_cb = a.n_tensors * a.units * (kHeadDim / rfft2::kCW);
+    const long long n_items = (long long)n_cb * (nA + nB);
+    long long grid = (long long)occ * ctx->n_sm;
+    if (grid > n_items) grid = n_items;
+    // pass B of a block is claimed `lag` blocks after its pass A: about the blocks the running CTAs span, plus one;
+    // the ring of the array between the passes holds twice that (and must hold more than the lag)
+    const size_t cb_bytes = ((size_t)1 << (LG1 + LG2)) * rfft2::kCP * sizeof(rfft2::C2);
+    long long ring_max = (long long)(f.yr_bytes / cb_bytes);
+    int lag = (int)((grid + nA - 1) / nA) + 1;
+    if (ring_max < 2) return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "two-pass array too small for the reconstruction ring");
+    if (lag > ring_max - 1) lag = (int)ring_max - 1;
+    if (lag > n_cb) lag = n_cb;
+    long long ring = 2LL * lag + 2;
+    if (ring > ring_max) ring = ring_max;
+    a.lag = lag;
+    a.ring = (int)ring;
+    kernel<<<(unsigned)grid, rfft2::kThreads, smem, st>>>(a);
+    return launch_check(ctx, "k_recon2");
+}
+
+template <typename TOut>
+int launch_recon2(faedkv_ctx *ctx, const LayerPlan &p, const float *coefK, const float *coefV, const int32_t *t_len, int units,
+                  int L, void *K_out, void *V_out, cudaStream_t st, ReconRows rows = ReconRows{0, -1, 0, 1}) {
+    if (rows.unit_rows < 0) rows.unit_rows = L;
+    const faedkv_config &c = ctx->cfg;
+    FftScratch &f = ctx->fs;
+    rfft2::Args a{};
+    a.n_tensors = 0;
+    if (coefK != nullptr) { a.coef[a.n_tensors] = coefK; a.out[a.n_tensors] = K_out; ++a.n_tensors; }
+    if (coefV != nullptr) { a.coef[a.n_tensors] = coefV; a.out[a.n_tensors] = V_out; ++a.n_tensors; }
+    a.units = units; a.M = p.M; a.H = c.n_kv_heads; a.Lrows = L;
+    a.slot = p.d_slot; a.t_len = t_len; a.tabP = f.r2_tabP; a.tabI = f.r2_tabI;
+    a.Y = reinterpret_cast<rfft2::C2 *>(f.Yr);
+    a.sync = f.r2_sync; a.status = ctx->dev_status; a.rows = rows;
+    const fft::Geometry g = fft::make_geometry(c.n_dft, kHeadDim);
+#define R2CASE(L1, L2, INST) if (g.lgN1 == L1 && g.lgN2 == L2) return launch_recon2_t<L1, L2, TOut>(ctx, a, INST, st)
+    R2CASE(3, 2, 0); R2CASE(3, 3, 1); R2CASE(4, 3, 2); R2CASE(4, 4, 3); R2CASE(5, 4, 4); R2CASE(5, 5, 5);
+    R2CASE(6, 5, 6); R2CASE(6, 6, 7); R2CASE(7, 6, 8); R2CASE(7, 7, 9); R2CASE(8, 7, 10); R2CASE(8, 8, 11);
+#undef R2CASE
+    return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "no reconstruction kernel for 2^%d x 2^%d points", g.lgN1, g.lgN2);
+}
+
 template <typename TOut>
 int launch_reconstruct_fft(faedkv_ctx *ctx, const LayerPlan &p, const float *coefK, const float *coefV, const int32_t *t_len,
                            int batch, int L, void *K_out, void *V_out, cudaStream_t st) {
     const int units = batch * ctx->cfg.n_kv_heads;
+    if (use_recon2(ctx))
+        return launch_recon2<TOut>(ctx, p, coefK, coefV, t_len, units, L, K_out, V_out, st);
     if (coefK != nullptr)
         if (int r = launch_reconstruct_fft_tensor<TOut>(ctx, p, coefK, t_len, units, L, K_out, st)) return r;
     if (coefV != nullptr)
@@ -932,6 +1020,7 @@ int faedkv_create(const faedkv_config *cfg, faedkv_ctx **out) {
         return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_sink < 0 || cfg->n_recent < 0 || cfg->n_sink + cfg->n_recent > 1024) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->n_defer < 0 || cfg->n_defer > 128) return FAEDKV_ERR_INVALID_ARG;
+    if (cfg->recon_engine < 0 || cfg->recon_engine > 2) return FAEDKV_ERR_INVALID_ARG;
     if (cfg->head_dim != kHeadDim) return FAEDKV_ERR_UNSUPPORTED;
     if (cfg->n_q_heads % cfg->n_kv_heads != 0) return FAEDKV_ERR_UNSUPPORTED;
     const int gq = cfg->n_q_heads / cfg->n_kv_heads;
@@ -1305,7 +1394,13 @@ int faedkv_reconstruct_windowed(faedkv_ctx *ctx, int layer, const float *coefK, 
     const int units = batch * c.n_kv_heads;
     // the reconstructed segment at rows [S, S + min(L - S, P)), zeros past its live positions ...
     const int Lmid = L - S < c.n_dft ? L - S : c.n_dft;
-    if (Lmid > 0) {
+    if (Lmid > 0 && use_recon2(ctx)) {
+        const ReconRows rows{S, L, -(S + R), D > 1 ? D : 1};
+        int r = c.kv_dtype == FAEDKV_BF16
+                    ? launch_recon2<__nv_bfloat16>(ctx, *p, coefK, coefV, t_len, units, Lmid, K_out, V_out, st, rows)
+                    : launch_recon2<float>(ctx, *p, coefK, coefV, t_len, units, Lmid, K_out, V_out, st, rows);
+        if (r) return r;
+    } else if (Lmid > 0) {
         const ReconRows rows{S, L, -(S + R), D > 1 ? D : 1};
         for (int kv = 0; kv < 2; ++kv) {
             const float *coef = kv == 0 ? coefK : coefV;

@@ -251,7 +251,12 @@ def test_checkpoint_restore_is_bit_exact(fk):
                                           (512, 100, 512, 1, 2, [512]), (96, 1, 50, 1, 1, [96]),
                                           (2048, 256, 2048, 1, 8, [2111]),      # config-0 shape after its 64 appends
                                           (8192, 64, 5001, 2, 3, [8192, 77]),   # two-pass split 64 x 64; odd L; ragged
-                                          (256, 129, 255, 1, 1, [256])])        # every bin retained
+                                          (256, 129, 255, 1, 1, [256]),         # every bin retained
+                                          # 24 column blocks of 128 x 128 points: more than the ring between the two
+                                          # passes holds, so ring slots are reused; odd L
+                                          (32768, 64, 20001, 1, 3, [32768]),
+                                          (131072, 32, 131072, 1, 1, [100000]),  # 256 x 256 points, the largest split
+                                          (64, 33, 64, 1, 2, [64])])            # the smallest grid: 8 x 4 points
 def test_reconstruct_matches_oracle(fk, oracle, dtype, P, M, L, B, H, tl):
     mask = _random_mask(P, M, 9 * P + L) if M > 1 else _mask_from_bins(P, [0])
     bins = oracle.plan(P, mask)
@@ -262,18 +267,25 @@ def test_reconstruct_matches_oracle(fk, oracle, dtype, P, M, L, B, H, tl):
     t_len = torch.from_numpy(t_np).cuda()
     wantK = oracle_reconstruct(oracle, to_np64(cK), P, bins, t_np, L)
     wantV = oracle_reconstruct(oracle, to_np64(cV), P, bins, t_np, L)
-    for mode in _decode_modes(fk, dtype, P):
+    modes = [(m, 0) for m in _decode_modes(fk, dtype, P)]
+    if P & (P - 1) == 0 and P >= 64:
+        modes.append((fk.DECODE_AUTO, 1))             # the FFT-shaped reconstruction's two engines, each forced:
+        if P <= (1 << 17):                            # a launch per pass, and the persistent kernel
+            modes.append((fk.DECODE_AUTO, 2))
+    if P > 16384:
+        modes = [m for m in modes if m[0] in (fk.DECODE_AUTO, fk.DECODE_FFT)]     # the dense evaluations are O(P M) per channel
+    for mode, engine in modes:
         ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=_kvd(fk, dtype),
-                         decode_mode=mode)
+                         decode_mode=mode, recon_engine=engine)
         ctx.plan(0, mask)
         Ko = torch.full((B, H, L, 128), 7.0, dtype=dtype, device="cuda")
         Vo = torch.full((B, H, L, 128), 7.0, dtype=dtype, device="cuda")
         ctx.reconstruct(0, cK, cV, t_len, L, Ko, Vo)
         torch.cuda.synchronize()
-        assert rel_l2(to_np64(Ko), wantK) <= _tol(dtype), mode
-        assert rel_l2(to_np64(Vo), wantV) <= _tol(dtype), mode
-        _rows_close(to_np64(Ko), wantK, _row_tol(dtype), ("token rows of K", mode))
-        _rows_close(to_np64(Vo), wantV, _row_tol(dtype), ("token rows of V", mode))
+        assert rel_l2(to_np64(Ko), wantK) <= _tol(dtype), (mode, engine)
+        assert rel_l2(to_np64(Vo), wantV) <= _tol(dtype), (mode, engine)
+        _rows_close(to_np64(Ko), wantK, _row_tol(dtype), ("token rows of K", mode, engine))
+        _rows_close(to_np64(Vo), wantV, _row_tol(dtype), ("token rows of V", mode, engine))
         for b in range(B):                                           # rows past the live length are exactly zero
             live = min(int(t_np[b]), P)
             if live < L:
