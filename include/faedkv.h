@@ -323,6 +323,28 @@ int faedkv_convert_state(faedkv_ctx *ctx, int layer, const float *coef_in, const
  * up.  Such a kernel returns early instead of hanging; its output is invalid. */
 int faedkv_device_status(faedkv_ctx *ctx, void *stream);
 
+/* Clear the device-side status word (enqueued on `stream`), so that a context whose kernel gave up a wait can be
+ * used, and watched, again. */
+int faedkv_reset_device_status(faedkv_ctx *ctx, void *stream);
+
+/* Test and diagnostics hooks of the tensor-core prefill (host state of the context; they apply to the calls
+ * that follow).  wait_limit_ns: time limit of each bounded mbarrier wait of that kernel (0 = the default,
+ * about one second).  withhold_step: 0 = off; s >= 1 = at pipeline step s (64 tokens per step) one producer
+ * warp of every CTA skips its "tile full" signal, so that every wait of the CTA runs out after wait_limit_ns:
+ * the kernel then records a code in the status word, waits for its own bulk copies, frees its tensor memory
+ * and returns -- the give-up path, exercised without any fault.  The output of such a call is invalid. */
+int faedkv_test_hooks(faedkv_ctx *ctx, unsigned long long wait_limit_ns, int withhold_step);
+
+/* Checked build.  The same sources compiled with -DFAEDKV_DEBUG (python -m paper_2507_20030_b200.build --debug
+ * -> lib/libfaedkv_debug.so) test every index that the kernels compute from data (bins, plan slots, ring
+ * slots, rows, tile offsets) against its bound before using it; a failed test records where it happened and
+ * skips the access, and the kernel returns normally.  faedkv_debug_build() is 1 in that build, else 0.
+ * faedkv_debug_word() synchronises `stream`, returns (file tag << 16 | source line) of the first failed test
+ * since the last call, or 0, and clears the word; it is always 0 in the normal build.  (The word is per
+ * process and device, not per context.) */
+int faedkv_debug_build(void);
+long long faedkv_debug_word(faedkv_ctx *ctx, void *stream);
+
 /* Decode attention for callers that cannot allocate -- the paper has no
  * counterpart; this is a packaging of faedkv_decode_attn() for hosts that
  * must not call cudaMalloc where they need it: code that runs while a CUDA

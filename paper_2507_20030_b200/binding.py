@@ -17,7 +17,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "lib", "libfaedkv.so")
+# FAEDKV_LIBRARY selects another build of the same library (the checked build, lib/libfaedkv_debug.so)
+LIB_PATH = os.environ.get("FAEDKV_LIBRARY") or os.path.join(_HERE, "lib", "libfaedkv.so")
 
 F32, BF16 = 0, 1
 PREFILL_AUTO, PREFILL_SIMT, PREFILL_UMMA, PREFILL_FFT = 0, 1, 2, 3
@@ -32,6 +33,7 @@ EXPORTS = [
     "faedkv_convert_state", "faedkv_window_bytes", "faedkv_prefill_windowed", "faedkv_step_windowed",
     "faedkv_reconstruct_windowed",
     "faedkv_device_status", "faedkv_launch_count", "faedkv_decode_attn_static",
+    "faedkv_reset_device_status", "faedkv_test_hooks", "faedkv_debug_build", "faedkv_debug_word",
 ]
 
 STATIC_SCRATCH_BYTES = 8 << 20
@@ -117,6 +119,14 @@ def load() -> ctypes.CDLL:
     lib.faedkv_decode_attn_static.restype = _int
     lib.faedkv_launch_count.argtypes = [_vp]
     lib.faedkv_launch_count.restype = ctypes.c_ulonglong
+    lib.faedkv_reset_device_status.argtypes = [_vp, _vp]
+    lib.faedkv_reset_device_status.restype = _int
+    lib.faedkv_test_hooks.argtypes = [_vp, ctypes.c_ulonglong, _int]
+    lib.faedkv_test_hooks.restype = _int
+    lib.faedkv_debug_build.argtypes = []
+    lib.faedkv_debug_build.restype = _int
+    lib.faedkv_debug_word.argtypes = [_vp, _vp]
+    lib.faedkv_debug_word.restype = ctypes.c_longlong
     _lib = lib
     return lib
 
@@ -360,3 +370,14 @@ class Context:
 
     def device_status(self, stream=None) -> int:
         return int(self._lib.faedkv_device_status(self._h, _stream(stream)))
+
+    def debug_word(self, stream=None) -> int:
+        """faedkv_debug_word: first failed bounds check of the checked build since the last call (0: none)."""
+        return int(self._lib.faedkv_debug_word(self._h, _stream(stream)))
+
+    def reset_device_status(self, stream=None):
+        self._check(self._lib.faedkv_reset_device_status(self._h, _stream(stream)))
+
+    def test_hooks(self, wait_limit_ns: int = 0, withhold_step: int = 0):
+        """faedkv_test_hooks: wait limit of the tensor-core prefill's bounded waits and the withheld-signal test."""
+        self._check(self._lib.faedkv_test_hooks(self._h, int(wait_limit_ns), int(withhold_step)))

@@ -9,6 +9,26 @@ namespace faedkv {
 
 constexpr int kHeadDim = 128;
 
+// Checked build (-DFAEDKV_DEBUG; stands in for a memory checker): an index computed from data -- a bin, a plan slot,
+// a ring slot, a row, a tile offset -- is tested against its bound before it addresses memory.  A failed test
+// records (file tag << 16 | source line) in a device word, once, and the access is skipped: the kernel carries
+// on and returns normally (never a trap), and the host reads the word with faedkv_debug_word().  In the normal
+// build the macro is the constant `true` and leaves no code behind.
+// Use:  if (!FAEDKV_IN_BOUNDS(tag, idx < n)) continue;   (or return, or skip the statement)
+#ifdef FAEDKV_DEBUG
+static __device__ unsigned int g_faedkv_debug_word = 0;
+__device__ __forceinline__ bool debug_in_bounds(bool ok, unsigned int where) {
+    if (!ok) atomicCAS(&g_faedkv_debug_word, 0u, where);
+    return ok;
+}
+#define FAEDKV_IN_BOUNDS(tag, cond) (::faedkv::debug_in_bounds((cond), ((unsigned int)(tag) << 16) | (unsigned int)__LINE__))
+#else
+#define FAEDKV_IN_BOUNDS(tag, cond) (true)
+#endif
+// file tags of FAEDKV_IN_BOUNDS
+constexpr unsigned int kTagAppend = 1, kTagAttnFft = 2, kTagAttnCol = 3, kTagRecon2 = 4, kTagPrefillUmma = 5,
+                       kTagDftSimt = 6, kTagWindow = 7, kTagFftEngine = 8, kTagReconFft = 9, kTagPrefillFft = 10;
+
 // (k * n) mod P with k, n < 2^31: the product fits 64 bits, so the reduced
 // phase index is exact however long the sequence is.
 __device__ __forceinline__ uint32_t phase_mod(uint32_t k, uint32_t n, uint32_t P) {

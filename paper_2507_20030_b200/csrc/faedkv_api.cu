@@ -9,6 +9,8 @@
 #include <string>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/faedkv.h"
 #include "common.cuh"
 #include "k_append.cuh"
@@ -28,6 +30,14 @@
 using namespace faedkv;
 
 namespace {
+
+// An NVTX range around a C-ABI call: names the call on a profiler's timeline; a no-op when no tool is attached.
+struct CallRange {
+    explicit CallRange(const char *name) { nvtxRangePushA(name); }
+    ~CallRange() { nvtxRangePop(); }
+    CallRange(const CallRange &) = delete;
+    CallRange &operator=(const CallRange &) = delete;
+};
 
 struct LayerPlan {
     int M = 0;
@@ -1070,6 +1080,7 @@ void faedkv_destroy(faedkv_ctx *ctx) {
 const char *faedkv_last_error(const faedkv_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
 int faedkv_plan(faedkv_ctx *ctx, int layer, const uint8_t *bin_mask, int *n_bins_out) {
+    const CallRange nvtx_range("faedkv_plan");
     if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;
     if (bin_mask == nullptr) return fail(ctx, FAEDKV_ERR_INVALID_ARG, "bin_mask is NULL");
     if (layer < 0 || layer >= ctx->cfg.n_layers)
@@ -1180,6 +1191,7 @@ int faedkv_mask_mixed(int n_dft, int n_keep, int layer, uint64_t seed, uint8_t *
 
 int faedkv_compress_prefill(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch,
                             int T, float *coefK, float *coefV, int32_t *t_len, void *stream) {
+    const CallRange nvtx_range("faedkv_compress_prefill");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1196,6 +1208,7 @@ int faedkv_compress_prefill(faedkv_ctx *ctx, int layer, const void *K, const voi
 
 int faedkv_append(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new, int batch,
                   float *coefK, float *coefV, int32_t *t_len, void *stream) {
+    const CallRange nvtx_range("faedkv_append");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1219,6 +1232,7 @@ int faedkv_append(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_n
 
 int faedkv_reconstruct(faedkv_ctx *ctx, int layer, const float *coefK, const float *coefV,
                        const int32_t *t_len, int batch, int L, void *K_out, void *V_out, void *stream) {
+    const CallRange nvtx_range("faedkv_reconstruct");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1243,6 +1257,7 @@ int faedkv_reconstruct(faedkv_ctx *ctx, int layer, const float *coefK, const flo
 
 int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *coefK, const float *coefV,
                        const int32_t *t_len, int batch, float scale, void *out, void *stream) {
+    const CallRange nvtx_range("faedkv_decode_attn");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1261,6 +1276,7 @@ int faedkv_decode_attn(faedkv_ctx *ctx, int layer, const void *q, const float *c
 int faedkv_append_decode_attn(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new, const void *q,
                               int batch, float *coefK, float *coefV, int32_t *t_len, float scale, void *out,
                               void *stream) {
+    const CallRange nvtx_range("faedkv_append_decode_attn");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1289,6 +1305,7 @@ size_t faedkv_window_bytes(const faedkv_ctx *ctx, int batch) {
 
 int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch, int T, float *coefK,
                             float *coefV, void *winK, void *winV, int32_t *t_len, void *stream) {
+    const CallRange nvtx_range("faedkv_prefill_windowed");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1331,6 +1348,7 @@ int faedkv_prefill_windowed(faedkv_ctx *ctx, int layer, const void *K, const voi
 int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const void *v_new, const void *q, int batch,
                          float *coefK, float *coefV, void *winK, void *winV, int32_t *t_len, float scale, void *out,
                          void *stream) {
+    const CallRange nvtx_range("faedkv_step_windowed");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1377,6 +1395,7 @@ int faedkv_step_windowed(faedkv_ctx *ctx, int layer, const void *k_new, const vo
 int faedkv_reconstruct_windowed(faedkv_ctx *ctx, int layer, const float *coefK, const float *coefV, const void *winK,
                                 const void *winV, const int32_t *t_len, int batch, int L, void *K_out, void *V_out,
                                 void *stream) {
+    const CallRange nvtx_range("faedkv_reconstruct_windowed");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1471,6 +1490,7 @@ int faedkv_mask_from_scores(int n_dft, int n_chunks, const double *delta, double
 
 int faedkv_ablate(faedkv_ctx *ctx, int layer, const void *K, const void *V, int batch, int T, const float *gain,
                   float *wsK, float *wsV, int32_t *ws_len, void *K_out, void *V_out, void *stream) {
+    const CallRange nvtx_range("faedkv_ablate");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1508,6 +1528,7 @@ int faedkv_ablate(faedkv_ctx *ctx, int layer, const void *K, const void *V, int 
 
 int faedkv_convert_state(faedkv_ctx *ctx, int layer, const float *coef_in, const int32_t *t_len, int batch, int from_form,
                          int to_form, float *coef_out, void *stream) {
+    const CallRange nvtx_range("faedkv_convert_state");
     const LayerPlan *p = nullptr;
     if (int r = check_layer(ctx, layer, &p)) return r;
     if (int r = check_batch(ctx, batch)) return r;
@@ -1526,6 +1547,43 @@ int faedkv_convert_state(faedkv_ctx *ctx, int layer, const float *coef_in, const
 }
 
 unsigned long long faedkv_launch_count(const faedkv_ctx *ctx) { return ctx ? ctx->launches : 0ULL; }
+
+int faedkv_reset_device_status(faedkv_ctx *ctx, void *stream) {
+    if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;
+    CUDA_TRY(ctx, cudaMemsetAsync(ctx->dev_status, 0, sizeof(unsigned int), static_cast<cudaStream_t>(stream)));
+    return FAEDKV_OK;
+}
+
+int faedkv_debug_build(void) {
+#ifdef FAEDKV_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+long long faedkv_debug_word(faedkv_ctx *ctx, void *stream) {
+    if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;
+#ifdef FAEDKV_DEBUG
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned int w = 0, zero = 0;
+    CUDA_TRY(ctx, cudaStreamSynchronize(st));
+    CUDA_TRY(ctx, cudaMemcpyFromSymbol(&w, g_faedkv_debug_word, sizeof(w)));
+    CUDA_TRY(ctx, cudaMemcpyToSymbol(g_faedkv_debug_word, &zero, sizeof(zero)));
+    if (w != 0) fail(ctx, FAEDKV_ERR_INVALID_ARG, "bounds check failed: file tag %u, line %u", w >> 16, w & 0xffffu);
+    return (long long)w;
+#else
+    (void)stream;
+    return 0;
+#endif
+}
+
+int faedkv_test_hooks(faedkv_ctx *ctx, unsigned long long wait_limit_ns, int withhold_step) {
+    if (ctx == nullptr || withhold_step < 0) return FAEDKV_ERR_INVALID_ARG;
+    ctx->umma.wait_limit_ns = wait_limit_ns == 0 ? umma::kWaitLimitNs : wait_limit_ns;
+    ctx->umma.withhold_step = withhold_step;
+    return FAEDKV_OK;
+}
 
 int faedkv_device_status(faedkv_ctx *ctx, void *stream) {
     if (ctx == nullptr) return FAEDKV_ERR_INVALID_ARG;

@@ -24,7 +24,7 @@ k_append(const TIn *__restrict__ k_new, const TIn *__restrict__ v_new, float *__
     const int b = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k = blockIdx.x * kAppendWarps + warp;
-    if (k < M) {
+    if (k < M && FAEDKV_IN_BOUNDS(kTagAppend, (uint32_t)bins[k] <= P / 2 && t_len[b] >= 0)) {
         const uint32_t t = (uint32_t)t_len[b];
         float c, s;
         twiddle(phase_mod((uint32_t)bins[k], t % P, P), P, c, s);

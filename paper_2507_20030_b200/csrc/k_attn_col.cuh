@@ -222,6 +222,7 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ bins,
     __syncthreads();
     for (int i = threadIdx.x; i < M; i += NT) {
         const int bin = bins[i];
+        if (!FAEDKV_IN_BOUNDS(kTagAttnCol, bin >= 0 && bin <= N)) continue;
         if (bin < N) {
             const float2 ph = tabP[bin];
             z[padded(bin)] = cmul(X[i], make_float2(1.f - ph.y, ph.x));          // 1 + j ph
@@ -230,6 +231,7 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ bins,
     __syncthreads();
     for (int i = threadIdx.x; i < M; i += NT) {
         const int bin = bins[i];
+        if (!FAEDKV_IN_BOUNDS(kTagAttnCol, bin >= 0 && bin <= N)) continue;
         if (bin > 0) {
             const int k = N - bin;
             const float2 ph = tabP[k];
@@ -271,6 +273,7 @@ k_afft_col(uint32_t P, int M, const int32_t *__restrict__ bins,
     float2 *out = Wg + (size_t)col * M;
     for (int i = threadIdx.x; i < M; i += NT) {
         const uint32_t bin = (uint32_t)bins[i];
+        if (!FAEDKV_IN_BOUNDS(kTagAttnCol, bin <= (uint32_t)N)) continue;
         const float w = 0.5f * hermitian_weight(bin, P) * f_col;
         const int ka = (int)bin & (N - 1), kb = (N - ka) & (N - 1);
         const float2 za = z[padded(ka)];

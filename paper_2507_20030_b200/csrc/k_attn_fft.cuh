@@ -102,6 +102,7 @@ k_attn_qs(const TQ *__restrict__ q, float *__restrict__ coefK, const TQ *__restr
         const bool self_conj = bin == 0u || 2u * bin == P;
         // Qs[bin][col] for the two-pass transforms, Qs[col][bin] for the one-kernel column transform
         const size_t col = (size_t)(b * HQ + h * GQ + g);
+        if (!FAEDKV_IN_BOUNDS(kTagAttnFft, bin <= P / 2 && col < (size_t)Gp)) return;
         float *dst = reinterpret_cast<float *>(Qs + (col_major ? col * M + (k0 + kk) : (size_t)(k0 + kk) * Gp + col));
         dst[pl] = (pl == 1 && self_conj) ? 0.f : tot * scale_over_P;
     }
@@ -412,7 +413,9 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
             const float w = 0.5f * hermitian_weight(bin, g.P);
             const int ka = (int)bin & (g.N - 1), kb = (g.N - ka) & (g.N - 1);
             const float2 ph = unit_phasor(bin, g.P);
-            const float2 *za_p = Zf + (uint32_t)ka * (uint32_t)g.Gp + gcol, *zb_p = Zf + (uint32_t)kb * (uint32_t)g.Gp + gcol;
+            // (checked build: a column outside the array reads column 0; no thread may leave before the barrier below)
+            const int zcol = FAEDKV_IN_BOUNDS(kTagAttnFft, bin <= g.P / 2 && gcol + GQ <= g.Gp) ? gcol : 0;
+            const float2 *za_p = Zf + (uint32_t)ka * (uint32_t)g.Gp + zcol, *zb_p = Zf + (uint32_t)kb * (uint32_t)g.Gp + zcol;
 #pragma unroll
             for (int q = 0; q < GQ; ++q) {
                 const float2 za = za_p[q];
@@ -473,7 +476,8 @@ k_attn_out_fft(float *__restrict__ coefV, const TQ *__restrict__ v_new, int32_t 
         float s = 0.f;
 #pragma unroll
         for (int w = 0; w < kAttnWarps; ++w) s += red[w][q][c];
-        partial[(((size_t)bh * slice_stride + blockIdx.x) * GQ + q) * kHeadDim + c] = s;
+        if (FAEDKV_IN_BOUNDS(kTagAttnFft, (int)blockIdx.x < slice_stride && bh < n_units))
+            partial[(((size_t)bh * slice_stride + blockIdx.x) * GQ + q) * kHeadDim + c] = s;
     }
     // last CTA of this (sequence, kv head): reduce the slices in a fixed order
     __threadfence();

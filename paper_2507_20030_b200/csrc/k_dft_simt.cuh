@@ -68,7 +68,8 @@ k_dft_forward_simt(DftUnitArgs a, const int32_t *__restrict__ bins, int M, uint3
 
     // twiddle generator: this thread owns bin gk and positions gj..gj+3 of every tile
     const int gk = tid & 31, gj = (tid >> 5) * 4;
-    const uint32_t gbin = (k0 + gk < M) ? (uint32_t)bins[k0 + gk] : 0u;
+    uint32_t gbin = (k0 + gk < M) ? (uint32_t)bins[k0 + gk] : 0u;
+    if (!FAEDKV_IN_BOUNDS(kTagDftSimt, gbin <= P / 2)) gbin = 0u;
     uint32_t ph[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) ph[i] = phase_mod(gbin, (pos0 + gj + i) % P, P);

@@ -190,8 +190,13 @@ __device__ __forceinline__ void fft_rows(int lg_cols_rt, float2 *xa, float2 *xb,
     constexpr int NF = 1 << LG;
     const int lg_cols = LGC >= 0 ? LGC : lg_cols_rt;
     constexpr int R1 = Radix<LG>::R1, R2 = Radix<LG>::R2, R3 = Radix<LG>::R3;
-    auto rd_a = [&](int row, int c) { return xa[(row << lg_cols) + c]; };
-    auto wr_a = [&](int row, int c, float2 v) { xa[(row << lg_cols) + c] = v; };
+    auto rd_a = [&](int row, int c) {
+        if (!FAEDKV_IN_BOUNDS(kTagFftEngine, row >= 0 && row < NF && c >= 0 && c < (1 << lg_cols))) return make_float2(0.f, 0.f);
+        return xa[(row << lg_cols) + c];
+    };
+    auto wr_a = [&](int row, int c, float2 v) {
+        if (FAEDKV_IN_BOUNDS(kTagFftEngine, row >= 0 && row < NF && c >= 0 && c < (1 << lg_cols))) xa[(row << lg_cols) + c] = v;
+    };
     auto rd_b = [&](int row, int c) { return xb[(row << lg_cols) + c]; };
     auto wr_b = [&](int row, int c, float2 v) { xb[(row << lg_cols) + c] = v; };
     if constexpr (R2 == 1) {

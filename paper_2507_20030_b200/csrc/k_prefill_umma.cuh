@@ -62,11 +62,13 @@ constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1
 }  // namespace prefill
 
 // grid = (ceil(M / 128), batch * H); block = 320; dynamic smem = Cfg<TERMS>::kSmemBytes
+// wait_limit_ns: time limit of every mbarrier wait; withhold_step: 0, or a test hook (see the generator loop)
 template <int TERMS>
 __global__ void __launch_bounds__(prefill::kThreads, 1)
 k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV,
                const int32_t *__restrict__ bins, int M, uint32_t P, int T, uint32_t pos0,
-               float *__restrict__ coefK, float *__restrict__ coefV, unsigned int *__restrict__ status) {
+               float *__restrict__ coefK, float *__restrict__ coefV, unsigned int *__restrict__ status,
+               unsigned long long wait_limit_ns, int withhold_step) {
     using namespace umma;
     using namespace prefill;
     using C = Cfg<TERMS>;
@@ -115,7 +117,7 @@ k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             for (int it = 0; it < n_steps && ok; ++it) {
                 const int s = it % S;
                 const uint32_t ph = (uint32_t)(it / S) & 1u;
-                if (!mbar_wait(empty(s), ph ^ 1u)) { ok = false; break; }
+                if (!mbar_wait(empty(s), ph ^ 1u, wait_limit_ns)) { ok = false; break; }
                 if (*abort_flag) break;
                 mbar_expect_tx(full_b(s), kBTileBytes);
                 const int n0 = it * kTileTok;
@@ -129,7 +131,7 @@ k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             if (!ok || *abort_flag) {
                 // wait (bounded) until the bulk copies still in flight have landed
                 for (int it = max(0, issued - S); it < issued; ++it)
-                    mbar_wait(full_b(it % S), (uint32_t)(it / S) & 1u);
+                    mbar_wait(full_b(it % S), (uint32_t)(it / S) & 1u, wait_limit_ns);
             }
         }
     } else if (warp == 1) {
@@ -139,7 +141,7 @@ k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             for (int it = 0; it < n_steps && ok; ++it) {
                 const int s = it % S;
                 const uint32_t ph = (uint32_t)(it / S) & 1u;
-                if (!mbar_wait(full_a(s), ph) || !mbar_wait(full_b(s), ph)) { ok = false; break; }
+                if (!mbar_wait(full_a(s), ph, wait_limit_ns) || !mbar_wait(full_b(s), ph, wait_limit_ns)) { ok = false; break; }
                 if (*abort_flag) break;
                 tc_fence_after();
 #pragma unroll
@@ -162,7 +164,8 @@ k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         const int g = threadIdx.x - 64;          // 0..255
         const int r = g & 127;                    // bin row of the tile
         const int hh = g >> 7;                    // which 32-token half of the stage
-        const uint32_t bin = (k0 + r < M) ? (uint32_t)bins[k0 + r] : 0u;
+        uint32_t bin = (k0 + r < M) ? (uint32_t)bins[k0 + r] : 0u;
+        if (!FAEDKV_IN_BOUNDS(kTagPrefillUmma, bin <= P / 2)) bin = 0u;
         float gc[8], gs[8];                       // e^{-jwk i}, i < 8: cos and sin of w k i
 #pragma unroll
         for (int i = 0; i < 8; ++i) twiddle(phase_mod(bin, (uint32_t)i % P, P), P, gc[i], gs[i]);
@@ -176,7 +179,7 @@ k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         for (int it = 0; it < n_steps; ++it) {
             const int s = it % S;
             const uint32_t ph = (uint32_t)(it / S) & 1u;
-            if (!mbar_wait(empty(s), ph ^ 1u)) { ok = false; break; }
+            if (!mbar_wait(empty(s), ph ^ 1u, wait_limit_ns)) { ok = false; break; }
             if (*abort_flag) break;
             float bc, bs;
             twiddle(ph_idx, P, bc, bs);
@@ -222,13 +225,15 @@ k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
             }
             fence_proxy_async();      // make the generic-proxy stores visible to the tensor core
             __syncwarp();
-            if (lane == 0) mbar_arrive(full_a(s));
+            // test hook (withhold_step > 0): the first generator warp skips its arrive at that step, so the tile never
+            // becomes "full" and every role's bounded wait runs out: the give-up path, exercised without a fault
+            if (lane == 0 && !(withhold_step > 0 && it == withhold_step - 1 && warp == 2)) mbar_arrive(full_a(s));
         }
         if (!ok) { atomicExch(status, kErrTimeoutGen); *abort_flag = 1; }
 
         // ---------------------------------------------------------------- epilogue (same 8 warps)
         bool have = ok && !*abort_flag;
-        if (have && !mbar_wait(accum_bar, 0u)) {
+        if (have && !mbar_wait(accum_bar, 0u, wait_limit_ns)) {
             have = false;
             atomicExch(status, kErrTimeoutEpi);
             *abort_flag = 1;
@@ -284,6 +289,8 @@ typedef CUresult (*PFN_encodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32
 struct UmmaPrefillState {
     PFN_encodeTiled encode = nullptr;
     bool attr_set[3] = {false, false, false};
+    unsigned long long wait_limit_ns = umma::kWaitLimitNs;   // test hooks: see faedkv_test_hooks()
+    int withhold_step = 0;
 };
 
 inline bool umma_prefill_available() { return true; }
@@ -337,7 +344,8 @@ inline int umma_launch_t(UmmaPrefillState &st, const CUtensorMap &mK, const CUte
         st.attr_set[TERMS] = true;
     }
     dim3 grid((M + prefill::kTileBinsU - 1) / prefill::kTileBinsU, units);
-    k_prefill_umma<TERMS><<<grid, prefill::kThreads, C::kSmemBytes, stream>>>(mK, mV, d_bins, M, (uint32_t)P, T, 0u, coefK, coefV, status);
+    k_prefill_umma<TERMS><<<grid, prefill::kThreads, C::kSmemBytes, stream>>>(mK, mV, d_bins, M, (uint32_t)P, T, 0u, coefK, coefV, status,
+                                                                              st.wait_limit_ns, st.withhold_step);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         snprintf(msg, n, "launch of k_prefill_umma failed: %s", cudaGetErrorString(e));

@@ -140,7 +140,9 @@ __device__ __forceinline__ void fft_rows(C2 *xa, const float2 *tw, Load load, St
     if constexpr (R2 == 1) {
         stage<NF, R1, 1, LGC>(tw, load, store);
     } else {
-        stage<NF, R1, 1, LGC>(tw, load, [&](int row, int c, C2 v) { xa[(row << LGC) + c] = v; });
+        stage<NF, R1, 1, LGC>(tw, load, [&](int row, int c, C2 v) {
+            if (FAEDKV_IN_BOUNDS(kTagRecon2, row >= 0 && row < NF && c >= 0 && c < (1 << LGC))) xa[(row << LGC) + c] = v;
+        });
         __syncthreads();
         stage<NF, R2, R1, LGC>(tw, [&](int row, int c) { return xa[(row << LGC) + c]; }, store);
     }
@@ -227,7 +229,6 @@ __global__ void __launch_bounds__(kThreads, min_ctas(LG1, LG2))
 k_recon2(Args a) {
     constexpr int N1 = 1 << LG1, N2 = 1 << LG2, N = N1 * N2;
     constexpr int LGKT = lg_per_tile(LG1, LG2), LGMT = lg_per_tile(LG2, LG1);
-    constexpr int KT = 1 << LGKT, MT = 1 << LGMT;
     constexpr int nA = N2 >> LGKT, nB = N1 >> LGMT;        // tiles per column block
     constexpr uint32_t P = 2u * N;
     extern __shared__ __align__(16) unsigned char smem2[];
@@ -268,6 +269,7 @@ k_recon2(Args a) {
         const int tile = isA ? idx : idx - nA;
         const int tensor = cb / (a.units * (kHeadDim / kCW)), cbu = cb % (a.units * (kHeadDim / kCW));
         const int unit = cbu / (kHeadDim / kCW), ch0 = (cbu % (kHeadDim / kCW)) * kCW;
+        if (!FAEDKV_IN_BOUNDS(kTagRecon2, cb >= 0 && cb < n_cb && tile >= 0 && tile < (isA ? nA : nB) && tensor < a.n_tensors)) continue;
         C2 *Yb = a.Y + (size_t)(cb % a.ring) * N * kCP;
         if (isA) {
             // the ring slot is free once pass B of the block that had it is through
@@ -281,6 +283,7 @@ k_recon2(Args a) {
                 const int cp = c & (kCP - 1), k = N2 * k1 + k2_0 + (c >> kLgCP);
                 const int sa = __ldg(a.slot + k), sb = __ldg(a.slot + (N - k));
                 // Z[k] = (X[k] + conj X[N-k]) + j e^{+j 2 pi k / P} (X[k] - conj X[N-k]);  bins 0 and N are real
+                if (!FAEDKV_IN_BOUNDS(kTagRecon2, sa < a.M && sb < a.M && k <= N)) return C2{make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 const float *pa = cu + (size_t)(sa < 0 ? 0 : sa) * kHeadDim + 2 * cp;
                 const float *pb = cu + (size_t)(sb < 0 ? 0 : sb) * kHeadDim + 2 * cp;
                 const float2 xr = ld_if(pa, sa >= 0), mr = ld_if(pb, sb >= 0);
@@ -315,6 +318,7 @@ k_recon2(Args a) {
             };
             auto store = [&](int m2, int c, C2 v) {
                 const int n = 2 * (m1_0 + (c >> kLgCP) + N1 * m2);
+                if (!FAEDKV_IN_BOUNDS(kTagRecon2, n >= 0 && n + 1 < (int)P + 1 && a.rows.row0 + (n < Lrows ? n : 0) < a.rows.unit_rows)) return;
                 TOut *o = obase + (size_t)n * kHeadDim + 2 * (c & (kCP - 1));
                 if (n < Lrows) { const bool lv = n < live; store_pair<TOut>(o, lv ? v.re.x : 0.f, lv ? v.re.y : 0.f); }
                 if (n + 1 < Lrows) { const bool lv = n + 1 < live; store_pair<TOut>(o + kHeadDim, lv ? v.im.x : 0.f, lv ? v.im.y : 0.f); }

@@ -49,7 +49,7 @@ k_rfft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float *__r
         const int col = g0 + c;
         float2 z = make_float2(0.f, 0.f);
         const int2 sl = tab_s[(k1 << lgKT) + kt];
-        if (sl.x >= 0 || sl.y >= 0) {
+        if ((sl.x >= 0 || sl.y >= 0) && FAEDKV_IN_BOUNDS(kTagReconFft, sl.x < M && sl.y < M)) {
             const float *u = coef + (size_t)(unit0 + (col >> 7)) * 2 * plane + (col & (kHeadDim - 1));
             float2 xk = make_float2(0.f, 0.f), xm = make_float2(0.f, 0.f);
             if (sl.x >= 0) xk = make_float2(u[(uint32_t)sl.x * kHeadDim], u[plane + (uint32_t)sl.x * kHeadDim]);

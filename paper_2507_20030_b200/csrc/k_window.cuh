@@ -17,7 +17,8 @@ struct FoldSrc {
 };
 __device__ __forceinline__ void fold_locate(const FoldSrc &f, int t, int unit, uint32_t P, size_t &row, uint32_t &pos) {
     if (f.R > 0) {
-        const int mid = t - f.S - f.R;                 // tokens already in the transformed segment
+        int mid = t - f.S - f.R;                       // tokens already in the transformed segment
+        if (!FAEDKV_IN_BOUNDS(kTagWindow, mid >= 0 && f.S + f.R <= f.unit_rows)) mid = 0;
         row = (size_t)unit * f.unit_rows + f.S + mid % f.R;
         pos = (uint32_t)mid % P;
     } else {

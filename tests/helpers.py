@@ -66,3 +66,29 @@ def oracle_decode_attn(orc, q: torch.Tensor, coefK: np.ndarray, coefV: np.ndarra
                 qn[b, h * G:(h + 1) * G], coefK[b, h, 0], coefK[b, h, 1], coefV[b, h, 0], coefV[b, h, 1],
                 P, bins, L, scale)
     return out
+
+
+class Guarded:
+    """A device tensor with a 256-byte canary before and after it: `t` is the tensor to hand to the library,
+    check() asserts that no byte outside it was written.  (The exact-zero and NaN fills of the parity tests catch
+    elements a kernel failed to write; this catches writes past either end.)"""
+    GUARD = 256
+    PATTERN = 0xA5
+
+    def __init__(self, shape, dtype, fill=None, device="cuda"):
+        n = 1
+        for s in shape:
+            n *= int(s)
+        nbytes = n * torch.empty((), dtype=dtype).element_size()
+        self.raw = torch.full((nbytes + 2 * self.GUARD,), self.PATTERN, dtype=torch.uint8, device=device)
+        self.t = self.raw[self.GUARD:self.GUARD + nbytes].view(dtype).view(*shape)
+        assert self.t.data_ptr() % 16 == 0
+        if fill is not None:
+            self.t.fill_(fill)
+        self.nbytes = nbytes
+
+    def check(self, what=""):
+        head = self.raw[:self.GUARD]
+        tail = self.raw[self.GUARD + self.nbytes:]
+        assert bool((head == self.PATTERN).all()), f"bytes before {what or 'the tensor'} were overwritten"
+        assert bool((tail == self.PATTERN).all()), f"bytes behind {what or 'the tensor'} were overwritten"

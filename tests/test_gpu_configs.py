@@ -176,14 +176,19 @@ def test_config3_long_context(fk, oracle):
 
 
 @pytest.mark.parametrize("T,B,r,mask_kind,layer", [
-    (4096, 32, 4, "lowpass", 0),
-    (16384, 8, 32, "mixed", 7),
     (4096, 1, 16, "mixed", 30),
+    (4096, 8, 4, "lowpass", 5),
+    (4096, 8, 32, "mixed", 11),
+    (4096, 32, 4, "lowpass", 0),
+    (16384, 1, 8, "mixed", 3),
+    (16384, 8, 32, "mixed", 7),
+    (16384, 8, 16, "lowpass", 20),
     (16384, 32, 8, "lowpass", 2),
 ])
 def test_config4_sweep_cells(fk, oracle, T, B, r, mask_kind, layer):
-    """configs[4]: Llama-2-7B-shaped MHA cache (32 kv = 32 query heads); corner cells of the
-    (T, batch, retention, mask) sweep, one layer each, prefill + 32 decode steps."""
+    """configs[4]: Llama-2-7B-shaped MHA cache (32 kv = 32 query heads); cells of the (T, batch, retention,
+    mask) sweep -- every (T, batch) pair, every retention ratio and both mask kinds occur -- one layer each,
+    prefill + 32 decode steps."""
     _decode_case(fk, oracle, config=4, layer=layer, B=B, H=32, HQ=32, T=T, M=T // r, mask_kind=mask_kind,
                  steps=32, sample_units=[(B - 1, 17)], sample_steps=[31])
 

@@ -775,6 +775,46 @@ def test_prefill_umma_matches_oracle(fk, oracle, terms, tol, P, T, M, B, H):
     ctx.close()
 
 
+def test_bounded_wait_gives_up_and_the_context_recovers(fk, oracle):
+    """The give-up path of the tensor-core prefill, run for real: with the wait limit at 1 ms and one producer's
+    'tile full' signal withheld at step 3, every wait of every CTA runs out; the kernel must end by itself (no
+    wait is unbounded), leave a code in the status word, and the next call on the same context, hooks off,
+    must be correct."""
+    import time
+    P = T = 1024
+    M, B, H = 200, 1, 3
+    ctx = fk.Context(n_layers=1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=fk.BF16,
+                     prefill_mode=fk.PREFILL_UMMA)
+    mask = _random_mask(P, M, 77)
+    ctx.plan(0, mask)
+    bins = oracle.plan(P, mask)
+    K, V = _make(12, B, H, T, torch.bfloat16)
+    cK, cV = ctx.alloc_coef(0, B), ctx.alloc_coef(0, B)
+    t_len = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    ctx.test_hooks(wait_limit_ns=1_000_000, withhold_step=3)
+    t0 = time.perf_counter()
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    torch.cuda.synchronize()
+    elapsed = time.perf_counter() - t0
+    assert elapsed < 1.0, elapsed                     # a handful of 1 ms waits, not the default second (nor forever)
+    code = ctx.device_status()
+    assert code in (0x11, 0x12, 0x13, 0x14), hex(code)   # one of the kernel's time-out codes
+    assert "bounded wait" in ctx._lib.faedkv_last_error(ctx._h).decode()
+    # hooks off, status cleared: the context works again
+    ctx.test_hooks(0, 0)
+    ctx.reset_device_status()
+    cK.fill_(float("nan")); cV.fill_(float("nan"))
+    ctx.compress_prefill(0, K.cuda(), V.cuda(), cK, cV, t_len)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    assert rel_l2(to_np64(cK), oracle_compress(oracle, K, P, bins)) <= REL_L2_BF16
+    assert rel_l2(to_np64(cV), oracle_compress(oracle, V, P, bins)) <= REL_L2_BF16
+    ctx.close()
+
+
 # ----------------------------------------------------------------------------- FFT-shaped prefill
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("P,T,M,B,H", [
