@@ -20,6 +20,7 @@
 #include "k_idft_umma.cuh"
 #include "k_attn_umma.cuh"
 #include "k_attn_fft.cuh"
+#include "k_attn_fft2.cuh"
 #include "k_attn_col.cuh"
 #include "k_recon_fft.cuh"
 #include "k_recon2.cuh"
@@ -70,6 +71,8 @@ struct FftScratch {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaStream_t side2 = nullptr;         // third stream: the second run of sequences of a call cut in two
     cudaEvent_t ev_cut = nullptr, ev_merge = nullptr;
+    float2 *a2_tabI = nullptr;            // inter-pass twiddles of the two-column attention transforms (P <= 2^17)
+    unsigned int a2_attr[3] = {0, 0, 0};  // their instances already opted in to large shared memory
     // second reconstruction engine (one persistent kernel; P <= 2^17)
     float2 *r2_tabP = nullptr, *r2_tabI = nullptr;
     unsigned int *r2_sync = nullptr;      // ticket, exit counter, per-column-block pass counters; zero between calls
@@ -185,7 +188,7 @@ void free_scratch(faedkv_ctx *ctx) {
     cudaFree(t.cmax); cudaFree(t.psum); cudaFree(t.colsum); cudaFree(t.PfS);
     t = TcScratch();
     FftScratch &f = ctx->fs;
-    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.o_win); cudaFree(f.Wg); cudaFree(f.colE); cudaFree(f.colB); cudaFree(f.colP); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr); cudaFree(f.r2_tabP); cudaFree(f.r2_tabI); cudaFree(f.r2_sync);
+    cudaFree(f.Qs); cudaFree(f.Y); cudaFree(f.Zf); cudaFree(f.mloc); cudaFree(f.sloc); cudaFree(f.colsum); cudaFree(f.o_win); cudaFree(f.Wg); cudaFree(f.colE); cudaFree(f.colB); cudaFree(f.colP); cudaFree(f.tickets); cudaFree(f.Yr); cudaFree(f.Zr); cudaFree(f.r2_tabP); cudaFree(f.r2_tabI); cudaFree(f.r2_sync); cudaFree(f.a2_tabI);
     if (f.side != nullptr) cudaStreamDestroy(f.side);
     if (f.ev_fork != nullptr) cudaEventDestroy(f.ev_fork);
     if (f.ev_join != nullptr) cudaEventDestroy(f.ev_join);
@@ -255,6 +258,8 @@ int ensure_scratch(faedkv_ctx *ctx, int M) {
                 CUDA_TRY(ctx, cudaMalloc(&f.r2_sync, n_sync * sizeof(unsigned int)));
                 CUDA_TRY(ctx, cudaMemset(f.r2_sync, 0, n_sync * sizeof(unsigned int)));
                 rfft2::k_recon2_tables<<<64, 256>>>(f.r2_tabP, f.r2_tabI, (uint32_t)c.n_dft, g.N2);
+                CUDA_TRY(ctx, cudaMalloc(&f.a2_tabI, (size_t)g.N * sizeof(float2)));
+                afft2::k_afft2_tables<<<64, 256>>>(f.a2_tabI, (uint32_t)g.N, g.N2);
                 CUDA_TRY(ctx, cudaDeviceSynchronize());
             }
             if (ctx->prefill_fft) CUDA_TRY(ctx, cudaMalloc(&f.Zr, ru * unit_bytes));
@@ -679,6 +684,44 @@ int launch_prefill_fft_tensor(faedkv_ctx *ctx, const LayerPlan &p, const void *x
     return FAEDKV_OK;
 }
 
+// Steps (2)-(4) through the two-column kernels (k_attn_fft2.cuh).  `join`: event to wait for before the last kernel
+// (the window statistics), or nullptr.
+template <int LG1, int LG2>
+int launch_afft2_t(faedkv_ctx *ctx, int inst, const fft::Geometry &g, const LayerPlan &p, const int32_t *t_len, int HQ, int t_add,
+                   int t_quant, int n_extra, cudaEvent_t join, cudaStream_t st) {
+    FftScratch &f = ctx->fs;
+    constexpr int lgKT = afft2::lg_per_tile(LG1, LG2), lgMT = afft2::lg_per_tile(LG2, LG1);
+    const afft2::Tables tb{f.r2_tabP, f.a2_tabI};
+    rfft2::C2 *Y2 = reinterpret_cast<rfft2::C2 *>(f.Y);
+    const int n_cb = g.Gp / afft2::kCW;
+    const unsigned int bit = 1u << inst;
+    constexpr size_t sa = afft2::smem_a<LG1, LG2>(), sm = afft2::smem_mid<LG1, LG2>(), sf = afft2::smem_fwd_b<LG1, LG2>();
+    if (sa > 48 * 1024 && !(f.a2_attr[0] & bit)) { if (int r = opt_in_smem(ctx, afft2::k_afft2_inv_a<LG1, LG2>, (uint32_t)sa)) return r; f.a2_attr[0] |= bit; }
+    if (sm > 48 * 1024 && !(f.a2_attr[1] & bit)) { if (int r = opt_in_smem(ctx, afft2::k_afft2_mid<LG1, LG2>, (uint32_t)sm)) return r; f.a2_attr[1] |= bit; }
+    if (sf > 48 * 1024 && !(f.a2_attr[2] & bit)) { if (int r = opt_in_smem(ctx, afft2::k_afft2_fwd_b<LG1, LG2>, (uint32_t)sf)) return r; f.a2_attr[2] |= bit; }
+    launch_pdl(afft2::k_afft2_inv_a<LG1, LG2>, dim3((1 << LG2) >> lgKT, n_cb), dim3(afft2::kThreads), sa, st, g.Gp, p.d_slot, f.Qs, tb, Y2);
+    if (int r = launch_check(ctx, "k_afft2_inv_a")) return r;
+    launch_pdl(afft2::k_afft2_mid<LG1, LG2>, dim3((1 << LG1) >> lgMT, n_cb), dim3(afft2::kThreads), sm, st, g.Gp, g.G, Y2, tb, t_len, HQ,
+               t_add, t_quant, f.mloc, f.sloc);
+    if (int r = launch_check(ctx, "k_afft2_mid")) return r;
+    if (join != nullptr) CUDA_TRY(ctx, cudaStreamWaitEvent(st, join, 0));
+    launch_pdl(afft2::k_afft2_fwd_b<LG1, LG2>, dim3((1 << LG2) >> lgKT, n_cb), dim3(afft2::kThreads), sf, st, g.Gp, Y2, tb, f.mloc, f.sloc,
+               f.Zf, f.colsum, n_extra);
+    return launch_check(ctx, "k_afft2_fwd_b");
+}
+
+// Whether the two-pass transforms of decode attention take the two-column kernels, and how many softmax tiles they make.
+bool use_afft2(const faedkv_ctx *ctx, const fft::Geometry &g) { return ctx->fs.a2_tabI != nullptr && g.lgN1 <= afft2::kMaxLg; }
+
+int launch_afft2(faedkv_ctx *ctx, const fft::Geometry &g, const LayerPlan &p, const int32_t *t_len, int HQ, int t_add, int t_quant,
+                 int n_extra, cudaEvent_t join, cudaStream_t st) {
+#define A2CASE(L1, L2, INST) if (g.lgN1 == L1 && g.lgN2 == L2) return launch_afft2_t<L1, L2>(ctx, INST, g, p, t_len, HQ, t_add, t_quant, n_extra, join, st)
+    A2CASE(3, 2, 0); A2CASE(3, 3, 1); A2CASE(4, 3, 2); A2CASE(4, 4, 3); A2CASE(5, 4, 4); A2CASE(5, 5, 5);
+    A2CASE(6, 5, 6); A2CASE(6, 6, 7); A2CASE(7, 6, 8); A2CASE(7, 7, 9); A2CASE(8, 7, 10); A2CASE(8, 8, 11);
+#undef A2CASE
+    return fail(ctx, FAEDKV_ERR_UNSUPPORTED, "no two-column transform for 2^%d x 2^%d points", g.lgN1, g.lgN2);
+}
+
 // FFT-shaped decode attention; with APPEND the IWDFT update of K and V rides on the two coefficient
 // streams and the token counters advance at the end.
 // A windowed step (winK != nullptr) folds the token leaving the recent ring instead of the new one, lets the
@@ -702,8 +745,9 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
     const int H = c.n_kv_heads, HQ = c.n_q_heads, M = p.M, P = c.n_dft;
     const fft::Geometry g = fft::make_geometry(P, batch * HQ);
     const int col_blocks = g.Gp / fft::kCW;
+    const bool two_col = !ctx->use_col && use_afft2(ctx, g);
     const int lgKT = fft::ilog2(fft::transforms_per_cta(g.N1, g.N2, col_blocks, ctx->n_sm));
-    const int lgMT = fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks, ctx->n_sm));
+    const int lgMT = two_col ? afft2::lg_per_tile(g.lgN2, g.lgN1) : fft::ilog2(fft::transforms_per_cta(g.N2, g.N1, col_blocks, ctx->n_sm));
     constexpr int KB = attn_bins_per_warp(GQ);
     // step (5) for the sequences [b0, b1) on stream s
     auto launch_out = [&](int b0, int b1, cudaStream_t s) -> int {
@@ -791,6 +835,8 @@ int launch_attn_fft(faedkv_ctx *ctx, const LayerPlan &p, const void *q, const vo
             CUDA_TRY(ctx, cudaStreamWaitEvent(st, f.ev_merge, 0));
         }
         rc = FAEDKV_OK;
+    } else if (two_col) {
+        if (int r = launch_afft2(ctx, g, p, t_len, HQ, (counts_new ? 1 : 0) - S - R, D, n_extra, n_extra ? f.ev_join : nullptr, st)) return r;
     } else {
     rc = FAEDKV_ERR_UNSUPPORTED;
     {

@@ -140,15 +140,13 @@ k_afft_inv_a(fft::Geometry g, const int32_t *__restrict__ slot, const float2 *__
     auto load = [&](int k1, int cidx) {
         const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;
         const int col = g0 + c;
-        float2 z = make_float2(0.f, 0.f);
+        // branch-free (see ld2_if): absent bins and padding columns read as zero
         const int2 sl = tab_s[(k1 << lgKT) + kt];
-        if ((sl.x >= 0 || sl.y >= 0) && col < g.G) {
-            const float2 xk = sl.x >= 0 ? Qs[(uint32_t)sl.x * (uint32_t)g.Gp + (uint32_t)col] : make_float2(0.f, 0.f);
-            float2 xm = sl.y >= 0 ? Qs[(uint32_t)sl.y * (uint32_t)g.Gp + (uint32_t)col] : make_float2(0.f, 0.f);
-            xm.y = -xm.y;                                            // conj X[N-k]
-            z = cadd(cadd(xk, xm), cmulj(cmul(tab_p[(k1 << lgKT) + kt], csub(xk, xm))));
-        }
-        return z;
+        const bool live_col = col < g.G;
+        const float2 xk = ld2_if(Qs + (uint32_t)(sl.x < 0 ? 0 : sl.x) * (uint32_t)g.Gp + (uint32_t)col, sl.x >= 0 && live_col);
+        float2 xm = ld2_if(Qs + (uint32_t)(sl.y < 0 ? 0 : sl.y) * (uint32_t)g.Gp + (uint32_t)col, sl.y >= 0 && live_col);
+        xm.y = -xm.y;                                                // conj X[N-k]
+        return cadd(cadd(xk, xm), cmulj(cmul(tab_p[(k1 << lgKT) + kt], csub(xk, xm))));
     };
     auto store = [&](int m1, int cidx, float2 v) {
         const int c = cidx & (kCW - 1), kt = cidx >> kLgCW;

@@ -36,7 +36,7 @@ __host__ __device__ constexpr int ilog2(int v) { return v <= 1 ? 0 : 1 + ilog2(v
 struct Geometry {
     uint32_t P;
     int N, N1, N2, lgN1, lgN2;
-    int Gp;        // allocated columns (multiple of kCW)
+    int Gp;        // allocated columns (multiple of 32: two column blocks of kCW, one of the two-column kernels)
     int G;         // real columns
 };
 inline Geometry make_geometry(int P, int G) {
@@ -49,7 +49,7 @@ inline Geometry make_geometry(int P, int G) {
     g.N1 = 1 << g.lgN1;
     g.N2 = 1 << g.lgN2;
     g.G = G;
-    g.Gp = (G + kCW - 1) / kCW * kCW;
+    g.Gp = (G + 31) / 32 * 32;
     return g;
 }
 // P is a power of two whose two passes fit the shared-memory tiles (3 <= lgN1 <= 9, 2 <= lgN2 <= 9).
@@ -70,6 +70,16 @@ __device__ __forceinline__ float2 cmul(float2 a, float2 b) {
 __device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
 __device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
 __device__ __forceinline__ float2 cmulj(float2 a) { return make_float2(-a.y, a.x); }   // j * a
+
+// Predicated global load: the value at p when pred, else zero, WITHOUT a branch.  The gathers of the half-spectrum
+// packing use it: behind branches every point of a butterfly waits for its own round trip to memory in turn;
+// predicated off instead of jumped over, the loads of all its points are in flight together.
+__device__ __forceinline__ float2 ld2_if(const float2 *p, bool pred) {
+    float2 v = make_float2(0.f, 0.f);
+    asm("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %3, 0;\n\t@q ld.global.v2.f32 {%0, %1}, [%2];\n\t}"
+        : "+f"(v.x), "+f"(v.y) : "l"(p), "r"((int)pred));
+    return v;
+}
 
 // e^{+j 2 pi num / den}, 0 <= num < den <= 2^24 (den a power of two: the quotient is exact).
 __device__ __forceinline__ float2 unit_phasor(uint32_t num, uint32_t den) {
