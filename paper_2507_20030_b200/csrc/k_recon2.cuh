@@ -325,6 +325,15 @@ k_recon2(Args a) {
             };
             fft_rows<LG2, LGMT + kLgCP>(xa, tw2, load, store);
             __syncthreads();                                // every read of the ring slot has returned
+            // The tile's part of the ring is dead now (pass A rewrites it whole before anyone reads it again): drop
+            // its lines from L2 instead of letting them be written back to DRAM when they are evicted.
+            {
+                const char *dead = reinterpret_cast<const char *>(Yb + (size_t)m1_0 * N2 * kCP);
+                constexpr int lines = (int)(((size_t)1 << LGMT) * N2 * kCP * sizeof(C2) / 128);
+                for (int i = threadIdx.x; i < lines; i += kThreads)
+                    asm volatile("discard.global.L2 [%0], 128;" ::"l"(dead + (size_t)i * 128) : "memory");
+            }
+            __syncthreads();
             if (threadIdx.x == 0) { __threadfence(); atomicAdd(doneB + cb, 1u); }
         }
     }
