@@ -51,6 +51,15 @@ WORKLOAD = dict(name="configs[1]: Llama-3-8B-shaped full cache, prefill 32768 to
                 M=4096, mask="mixed")
 
 
+def workload_config(W, prefill_path, twiddle_terms):
+    """The `config` object of a bench line (both arms print the same one for the same workload)."""
+    return {"workload": W["name"], "n_layers": W["n_layers"], "n_kv_heads": W["n_kv_heads"], "n_q_heads": W["n_q_heads"],
+            "head_dim": W["head_dim"], "batch": W["batch"], "T": W["T"], "n_dft": W["T"], "n_bins": W["M"],
+            "mask": "mixed (seeded, per layer)", "prefill_path": prefill_path, "twiddle_terms": twiddle_terms,
+            "l2": "inputs larger than L2: 32 layers cycled, 128 MiB K/V + 64 MiB planes per layer",
+            "multi_gpu": "replicas only"}
+
+
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -265,7 +274,8 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": W["name"], "extrapolated": True},
+            "config": workload_config(W, "tcgen05-bf16", 1),     # the same workload description as our arm's line
+            "extrapolated": True,
             "cpu_baseline": {**base, "value": v},
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -474,6 +484,54 @@ def decode_section(torch, binding, synth, dev, W, peaks, iters, graphs=True):
     del cKs, cVs
     torch.cuda.empty_cache()
     return res
+
+
+# --------------------------------------------------------------------------------------- configs[0]
+def config0_section(torch, binding, synth, dev):
+    """configs[0] on the GPU as it is stated: 1 layer, 8 kv heads, 2048 float32 tokens, 256 low-pass bins; prefill, 64
+    appends, reconstruct (L = 2048).  Its planes (8 MiB) sit in L2, so only times are reported, no bandwidth
+    fraction; the oracle's times for the same work are under cpu_baseline.config0_full."""
+    P = T = 2048
+    M, H, HQ, steps = 256, 8, 32, 64
+    seed = synth.config_seed(0, 0)
+    ctx = binding.Context(n_layers=1, n_kv_heads=H, n_q_heads=HQ, n_dft=P, max_batch=1, kv_dtype=binding.F32)
+    ctx.plan(0, binding.mask_lowpass(P, M))
+    K, V = synth.make_kv(seed, 1, H, T, 128, dtype=torch.float32, device=dev)
+    toks = [synth.make_token(seed, s_, 1, H, 128, pos=T + s_, dtype=torch.float32, device=dev) for s_ in range(steps)]
+    cK, cV = ctx.alloc_coef(0, 1, device=dev), ctx.alloc_coef(0, 1, device=dev)
+    tl = torch.zeros(1, dtype=torch.int32, device=dev)
+    Ko = torch.empty((1, H, P, 128), dtype=torch.float32, device=dev)
+    Vo = torch.empty_like(Ko)
+
+    def run():
+        ctx.compress_prefill(0, K, V, cK, cV, tl)
+        for k, v in toks:
+            ctx.append(0, k, v, cK, cV, tl)
+        ctx.reconstruct(0, cK, cV, tl, P, Ko, Vo)
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    reps = 10
+    tp = ta = tr = 0.0
+    for _ in range(reps):
+        ev[0].record()
+        ctx.compress_prefill(0, K, V, cK, cV, tl)
+        ev[1].record()
+        for k, v in toks:
+            ctx.append(0, k, v, cK, cV, tl)
+        ev[2].record()
+        ctx.reconstruct(0, cK, cV, tl, P, Ko, Vo)
+        ev[3].record()
+        torch.cuda.synchronize()
+        tp += ev[0].elapsed_time(ev[1]); ta += ev[1].elapsed_time(ev[2]); tr += ev[2].elapsed_time(ev[3])
+    if ctx.device_status() != 0:
+        raise RuntimeError("a kernel reported a device-side timeout; the numbers are invalid")
+    ctx.close()
+    return {"workload": "configs[0]: 1 layer, batch 1, 8 kv heads, 2048 float32 tokens, 256 low-pass bins, 64 appends, reconstruct",
+            "prefill_us": tp / reps * 1e3, "prefill_tokens_per_s": T / (tp / reps * 1e-3), "prefill_path": "FFT-shaped float32 (default for float32 K/V)",
+            "append_us_per_step": ta / reps / steps * 1e3, "reconstruct_us": tr / reps * 1e3, "total_us": (tp + ta + tr) / reps * 1e3,
+            "launch": "eager, CUDA events around each phase; planes are L2-resident (8 MiB)"}
 
 
 # --------------------------------------------------------------------------------------- configs[4] sweep
@@ -785,6 +843,9 @@ def run_ours(args):
         torch.cuda.empty_cache()
         for DW in DECODE_WORKLOADS:
             decode_sections.append(decode_section(torch, binding, synth, dev, DW, peaks, args.decode_config_iters))
+    config0 = None
+    if not args.no_decode_configs and not args.layers:
+        config0 = config0_section(torch, binding, synth, dev)
     sweep = None
     if not args.no_sweep and not args.no_decode_configs and not args.layers:
         cells = sweep_cells()
@@ -855,13 +916,10 @@ def run_ours(args):
     line = {"metric": METRIC, "value": whole_job_value(B * T, world, prefill_ms), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": W["name"], "n_layers": NL, "n_kv_heads": H, "n_q_heads": HQ, "head_dim": D,
-                       "batch": B, "T": T, "n_dft": P, "n_bins": M, "mask": "mixed (seeded, per layer)",
-                       "prefill_path": mode, "twiddle_terms": args.twiddle_terms or 1,
-                       "l2": "inputs larger than L2: 32 layers cycled, 128 MiB K/V + 64 MiB planes per layer",
-                       "multi_gpu": "replicas only"},
+            "config": workload_config(W, mode, args.twiddle_terms or 1),
             "phase_ms": phase_ms, "prefill_ms": prefill_ms,
             "roofline": roofline, "prefill_fft": prefill_fft, "decode": decode, "e2e": e2e, "gpu_launches": launches, "clocks": clocks}
+    line["config0"] = config0
     line["sweep"] = sweep
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline()
@@ -880,6 +938,9 @@ def run_ours(args):
                         "win": pair(sec["step_windowed"]), "defer": pair(sec["step_windowed_deferred"])}
         if "reconstruct" in sec:
             summary[key]["recon"] = pair(sec["reconstruct"])
+    if config0 is not None:
+        summary["cfg0"] = {"prefill_us": round(config0["prefill_us"], 1), "append_us": round(config0["append_us_per_step"], 2),
+                           "recon_us": round(config0["reconstruct_us"], 1)}
     line["decode_summary"] = summary
     print(json.dumps(line))
     if world > 1:
