@@ -17,7 +17,8 @@
 // Twiddle precision: every twiddle is the product of three float32 unit
 // phasors whose angles come from exactly reduced integer phases
 //     e^{-jwk(n0 + 8c + i)} = e^{-jwk n0} * (e^{-jwk 8})^c * e^{-jwk i},
-// (absolute error < 1e-6), then rounded to bf16 once (TERMS = 1, relative
+// where the stage base e^{-jwk n0} is re-derived from the integer phase every 16th stage and rotated by
+// e^{-jwk 64} in between (absolute error < 1e-6), then rounded to bf16 once (TERMS = 1, relative
 // error of a coefficient ~1e-3) or split into a bf16 hi + lo pair (TERMS = 2,
 // ~1e-5, twice the MMA work).  Accumulation is float32 in TMEM.
 //
@@ -169,28 +170,49 @@ k_prefill_umma(const __grid_constant__ CUtensorMap mapK, const __grid_constant__
         float gc[8], gs[8];                       // e^{-jwk i}, i < 8: cos and sin of w k i
 #pragma unroll
         for (int i = 0; i < 8; ++i) twiddle(phase_mod(bin, (uint32_t)i % P, P), P, gc[i], gs[i]);
+        // the same as pairs (i, i + 1), for the packed float32x2 form of the rotation below
+        float2 gc2[4], gs2[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { gc2[j] = make_float2(gc[2 * j], gc[2 * j + 1]); gs2[j] = make_float2(gs[2 * j], gs[2 * j + 1]); }
         float f1c, f1s;                           // cos, sin of w k 8
         twiddle(phase_mod(bin, 8u % P, P), P, f1c, f1s);
         uint32_t ph_idx = phase_mod(bin, (pos0 + (uint32_t)hh * 32u) % P, P);
         const uint32_t step_idx = phase_mod(bin, (uint32_t)kTileTok % P, P);
         const uint32_t row_off = (uint32_t)r * 128u;
         const uint32_t sw = (uint32_t)(r & 7);
+        float stc, sts;                           // cos, sin of w k 64: one stage further
+        twiddle(step_idx, P, stc, sts);
+        float base_c = 1.f, base_s = 0.f;         // phasor of the first token this thread writes in the current stage
         bool ok = true;
         for (int it = 0; it < n_steps; ++it) {
             const int s = it % S;
             const uint32_t ph = (uint32_t)(it / S) & 1u;
             if (!mbar_wait(empty(s), ph ^ 1u, wait_limit_ns)) { ok = false; break; }
             if (*abort_flag) break;
-            float bc, bs;
-            twiddle(ph_idx, P, bc, bs);
+            // every 16th stage the base phasor comes from the exactly reduced integer phase; in between it is rotated
+            // one stage forward (15 float32 rotations at most: error < 1e-6, nothing accumulates beyond that)
+            if ((it & 15) == 0) {
+                twiddle(ph_idx, P, base_c, base_s);
+            } else {
+                const float nc = fmaf(base_c, stc, -base_s * sts);
+                base_s = fmaf(base_s, stc, base_c * sts);
+                base_c = nc;
+            }
+            float bc = base_c, bs = base_s;
             ph_idx = add_mod(ph_idx, step_idx, P);
 #pragma unroll
             for (int cc = 0; cc < 4; ++cc) {
+                // cos(a + b) = bc gc - bs gs, sin(a + b) = bs gc + bc gs for two tokens per instruction: the packed
+                // FMA rounds each lane exactly like fmaf(bc, gc, -bs * gs), at half the instructions (the generator
+                // warps' arithmetic is the part of this kernel's power that is not the tensor core's)
                 float vc[8], vs[8];
+                const float2 bc2 = make_float2(bc, bc), bs2 = make_float2(bs, bs), nbs2 = make_float2(-bs, -bs);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    vc[i] = fmaf(bc, gc[i], -bs * gs[i]);     // cos(a + b)
-                    vs[i] = fmaf(bs, gc[i], bc * gs[i]);      // sin(a + b)
+                for (int j = 0; j < 4; ++j) {
+                    const float2 c2 = __ffma2_rn(bc2, gc2[j], __fmul2_rn(nbs2, gs2[j]));
+                    const float2 s2 = __ffma2_rn(bs2, gc2[j], __fmul2_rn(bc2, gs2[j]));
+                    vc[2 * j] = c2.x; vc[2 * j + 1] = c2.y;
+                    vs[2 * j] = s2.x; vs[2 * j + 1] = s2.y;
                 }
                 const uint32_t chunk = (((uint32_t)(hh * 4 + cc)) ^ sw) << 4;
                 uint4 pc, psn;
