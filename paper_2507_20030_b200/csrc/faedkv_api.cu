@@ -176,10 +176,6 @@ int out_slices(const faedkv_ctx *ctx, int batch, int M) {
     int cap = (M + 63) / 64;
     if (s > cap) s = cap;
     if (s < 1) s = 1;
-    // a slice of more than one chunk of bins (kOutChunk) pays the weight prologue twice and ends in a short chunk:
-    // take one-chunk slices instead while their CTAs still fit the GPU in one wave (4 per SM)
-    const int per = (M + s - 1) / s, s1 = (M + kOutChunk - 1) / kOutChunk;
-    if (per > kOutChunk && (long long)s1 * units <= 4LL * ctx->n_sm && s1 <= ctx->out_slices_cap) s = s1;
     return s;
 }
 
