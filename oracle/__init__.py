@@ -63,6 +63,7 @@ def _load():
         "orc_compress_units": (None, [_f64p, _int, _int, _int, _int, _i32p, _int, _i64, _f64p, _f64p]),
         "orc_append": (None, [_f64p, _f64p, _int, _int, _int, _i32p, _i64, _f64p]),
         "orc_reconstruct": (None, [_f64p, _f64p, _int, _int, _int, _i32p, _int, _f64p]),
+        "orc_reconstruct_rows": (None, [_f64p, _f64p, _int, _int, _int, _i32p, _i32p, _int, _f64p]),
         "orc_attention_dense": (None, [_f64p, _int, _f64p, _f64p, _int, _int, _f64, _f64p]),
         "orc_decode_attn": (None, [_f64p, _int, _f64p, _f64p, _f64p, _f64p, _int, _int, _int,
                                    _i32p, _int, _f64, _f64p]),
@@ -175,6 +176,17 @@ def reconstruct(Cre: np.ndarray, Cim: np.ndarray, P: int, bins: np.ndarray, L: i
     M, d = Cre.shape
     out = np.zeros((L, d), dtype=np.float64)
     _load().orc_reconstruct(_d(Cre), _d(Cim), M, d, P, _i(bins), L, _d(out))
+    return out
+
+
+def reconstruct_rows(Cre: np.ndarray, Cim: np.ndarray, P: int, bins: np.ndarray, rows) -> np.ndarray:
+    """Pruned inverse DFT of one unit's planes at the listed positions only -> [len(rows), d]."""
+    bins = np.ascontiguousarray(bins, dtype=np.int32)
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    Cre, Cim = _f64arr(Cre), _f64arr(Cim)
+    M, d = Cre.shape
+    out = np.zeros((rows.shape[0], d), dtype=np.float64)
+    _load().orc_reconstruct_rows(_d(Cre), _d(Cim), M, d, P, _i(bins), _i(rows), int(rows.shape[0]), _d(out))
     return out
 
 

@@ -199,6 +199,26 @@ void orc_reconstruct(const double *Cre, const double *Cim, int M, int d, int P,
     }
 }
 
+/* The same sum at the listed positions only: out[i,c] = xtilde[rows[i], c].  (Eq. 5 on the retained bins,
+ * position by position; lets a caller check single rows of a long reconstruction.) */
+void orc_reconstruct_rows(const double *Cre, const double *Cim, int M, int d, int P,
+                          const int32_t *bins, const int32_t *rows, int n_rows, double *out) {
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < n_rows; ++i) {
+        const int64_t n = rows[i];
+        double *o = out + (size_t)i * d;
+        for (int c = 0; c < d; ++c) o[c] = 0.0;
+        for (int ki = 0; ki < M; ++ki) {
+            double a = phase_angle(phase_index(bins[ki], n, P), P);
+            double w = orc_weight(P, bins[ki]);
+            double co = w * cos(a), si = w * sin(a);
+            const double *re = Cre + (size_t)ki * d, *im = Cim + (size_t)ki * d;
+            for (int c = 0; c < d; ++c) o[c] += re[c] * co - im[c] * si;
+        }
+        for (int c = 0; c < d; ++c) o[c] /= (double)P;
+    }
+}
+
 /* ------------------------------------------------------ O5: decode attention (Eq. 3 on Eq. 11) */
 
 /* Textbook single-query attention on the materialised reconstruction:

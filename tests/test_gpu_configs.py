@@ -245,3 +245,56 @@ def test_config2_windowed_workflow(fk, oracle, defer):
             err = rel_l2(to_np64(c[b, h]), np.stack(want))
             assert err <= REL_L2_BF16, ("planes", b, h, err)
     ctx.close()
+
+
+@pytest.mark.parametrize("config,B,H,T,M,tl_short", [
+    (1, 1, 8, 32768, 4096, None),          # one persistent launch, 64 column blocks
+    (2, 16, 8, 16384, 2048, 9000),         # 1024 column blocks: the ring between the passes is reused 50 times over
+    (3, 1, 8, 131072, 8192, None),         # the two-kernel engine (256-point passes)
+])
+def test_reconstruct_full_sizes(fk, oracle, config, B, H, T, M, tl_short):
+    """Reconstruction at the full sizes of configs[1], [2] and [3], in the launch configuration the benchmark
+    times (bf16 rows, default engine): both tensors written whole, then single rows of sampled units compared
+    with the oracle's row-wise inverse transform -- first and last rows, rows around tile and pass boundaries,
+    rows around the live length of a shorter sequence, random rows."""
+    from paper_2507_20030_b200 import synth
+    P, layer = T, 5
+    seed = synth.config_seed(config)
+    ctx = fk.Context(n_layers=layer + 1, n_kv_heads=H, n_q_heads=H, n_dft=P, max_batch=B, kv_dtype=fk.BF16)
+    mask = fk.mask_mixed(P, M, layer, seed)
+    ctx.plan(layer, mask)
+    bins = oracle.plan(P, oracle.mask_mixed(P, M, layer, seed))
+    g = torch.Generator(device="cuda").manual_seed(seed + 17)
+    # planes with the decaying spectrum of a real cache (large low bins), random phases
+    amp = (float(np.sqrt(T)) / (1.0 + torch.arange(M, device="cuda", dtype=torch.float32) / 64.0))[None, None, None, :, None]
+    cK = torch.randn((B, H, 2, M, D), generator=g, device="cuda") * amp
+    cV = torch.randn((B, H, 2, M, D), generator=g, device="cuda") * amp
+    tl = np.full(B, T + 3, dtype=np.int32)
+    if tl_short is not None:
+        tl[B // 2] = tl_short
+    t_len = torch.from_numpy(tl).cuda()
+    Ko = torch.full((B, H, P, D), 7.0, dtype=torch.bfloat16, device="cuda")
+    Vo = torch.full_like(Ko, 7.0)
+    ctx.reconstruct(layer, cK, cV, t_len, P, Ko, Vo)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    rng = np.random.default_rng(config)
+    N1 = 1 << ((P // 2).bit_length() // 2)
+    special = [0, 1, 2, 3, 2 * N1 - 2, 2 * N1 - 1, 2 * N1, 2 * N1 + 1, P // 2 - 1, P // 2, P // 2 + 1, P - 2, P - 1]
+    units = sorted({(0, 0), (B - 1, H - 1), (B // 2, H // 2), (B // 2, 0)})
+    for b, h in units:
+        live = min(int(tl[b]), P)
+        rows = sorted(set(special + list(rng.integers(0, P, size=40)) +
+                          ([live - 2, live - 1, live, live + 1] if live < P else [])))
+        rows = np.array([r for r in rows if 0 <= r < P], dtype=np.int32)
+        for c, X in ((cK, Ko), (cV, Vo)):
+            pl = to_np64(c[b, h])
+            want = oracle.reconstruct_rows(pl[0], pl[1], P, bins, rows)
+            want[rows >= live] = 0.0
+            got = to_np64(X[b, h][torch.from_numpy(rows.astype(np.int64)).cuda()])
+            assert not got[rows >= live].any(), (b, h)                       # rows past the live length are exactly zero
+            scale = np.sqrt((want ** 2).sum(axis=1).mean())
+            err = np.sqrt(((got - want) ** 2).sum(axis=1)).max() / scale     # worst row against the typical row norm
+            assert err <= 4 * REL_L2_BF16, (config, b, h, err)
+            assert rel_l2(got, want) <= REL_L2_BF16, (config, b, h, rel_l2(got, want))
+    ctx.close()

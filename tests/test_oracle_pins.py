@@ -294,6 +294,26 @@ def test_all_bins_attention_is_textbook(oracle, P, t):
     np.testing.assert_allclose(out2, _textbook_attention(q, K, V, 0.37), atol=1e-12)
 
 
+def test_reconstruct_rows_is_the_inverse_transform_at_those_rows(oracle):
+    """Row-wise reconstruction: with every bin kept it returns the input rows themselves (and x[n mod P] beyond P,
+    the sum being P-periodic); with a pruned set it equals numpy's irfft of the zero-filled half spectrum."""
+    P, d = 48, 5
+    rng = _rng(77)
+    x = rng.standard_normal((P, d))
+    bins = _all_bins(P)
+    cr, ci = oracle.compress(x, P, bins)
+    rows = np.array([0, 1, 17, 47, 46, 5], dtype=np.int32)
+    np.testing.assert_allclose(oracle.reconstruct_rows(cr, ci, P, bins, rows), x[rows], atol=1e-12)
+    np.testing.assert_allclose(oracle.reconstruct_rows(cr, ci, P, bins, rows + P), x[rows], atol=1e-12)
+    keep = np.array([0, 2, 3, 7, 24], dtype=np.int32)               # includes both self-conjugate bins
+    kr, ki = oracle.compress(x, P, keep)
+    half = np.zeros((P // 2 + 1, d), dtype=complex)
+    half[keep] = kr + 1j * ki
+    want = np.fft.irfft(half, n=P, axis=0)
+    np.testing.assert_allclose(oracle.reconstruct_rows(kr, ki, P, keep, rows), want[rows], atol=1e-12)
+    np.testing.assert_allclose(oracle.reconstruct(kr, ki, P, keep, P)[rows], want[rows], atol=1e-12)
+
+
 def test_attention_over_no_token_is_zero(oracle):
     """L = 0: Eq. 3 has no token to sum over; the reading taken is the empty sum, a zero vector (never NaN),
     and one token gives that token's value row whatever the query."""
